@@ -1,0 +1,146 @@
+"""ctypes front end of the CPU oracle (TEST INFRASTRUCTURE, not a product path).
+
+Only the tests, the smoke check and the benchmark's cpu-baseline leg may import this package.
+It compiles ``sgo.c`` with gcc on first use and marshals numpy arrays; all arithmetic is in the C
+file.  bf16 tensors travel as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sgo.c")
+_LIB = os.path.join(_HERE, "libsgo.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (gcc -O2 -fopenmp) next to its source; returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.sgo_max_threads.restype = ctypes.c_int
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().sgo_max_threads())
+
+
+def set_threads(n: int) -> None:
+    _load().sgo_set_threads(ctypes.c_int(int(n)))
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.asarray(a)
+    if a.dtype != dtype:
+        raise TypeError("expected %s, got %s" % (np.dtype(dtype), a.dtype))
+    return np.ascontiguousarray(a)
+
+
+def _i64(x):
+    return ctypes.c_int64(int(x))
+
+
+def score(q_win: np.ndarray, k_cache: np.ndarray, cu_seqlens: np.ndarray, window: Optional[int] = None) -> np.ndarray:
+    """importance float32 [L][H_kv][T] from q_win uint16 [L][B][W][H_q][d] and k_cache uint16 [L][T][H_kv][d]."""
+    q_win, k_cache, cu = _c(q_win, np.uint16), _c(k_cache, np.uint16), _c(cu_seqlens, np.int32)
+    L, B, W, Hq, d = q_win.shape
+    L2, T, Hkv, d2 = k_cache.shape
+    assert L == L2 and d == d2 and cu.shape == (B + 1,) and cu[-1] == T
+    assert window is None or window == W
+    imp = np.zeros((L, Hkv, T), dtype=np.float32)
+    rc = _load().sgo_score(L, B, Hq, Hkv, d, W, _p(cu), _p(q_win), _p(k_cache),
+                           _i64(T * Hkv * d), _i64(Hkv * d), _i64(d), _p(imp))
+    if rc:
+        raise RuntimeError("sgo_score failed: %d" % rc)
+    return imp
+
+
+def select_topk(importance: np.ndarray, cu_seqlens: np.ndarray, cu_k: np.ndarray) -> np.ndarray:
+    """sel_idx int32 [L][H_kv][K_tot] (ascending, sequence-local) from importance float32 [L][H_kv][T]."""
+    imp, cu, ck = _c(importance, np.float32), _c(cu_seqlens, np.int32), _c(cu_k, np.int32)
+    L, Hkv, T = imp.shape
+    B = cu.shape[0] - 1
+    assert cu[-1] == T and ck.shape == (B + 1,)
+    sel = np.zeros((L, Hkv, int(ck[-1])), dtype=np.int32)
+    rc = _load().sgo_select_topk(L, B, Hkv, _p(cu), _p(imp), _p(ck), _p(sel))
+    if rc:
+        raise RuntimeError("sgo_select_topk failed: %d" % rc)
+    return sel
+
+
+def pack_kv(k_cache: np.ndarray, v_cache: np.ndarray, cu_seqlens: np.ndarray, sel_idx: np.ndarray, cu_k: np.ndarray):
+    """packed_k, packed_v uint16 [L][K_tot*H_kv][d]; row of (b, g, j) is cu_k[b]*H_kv + g*k_b + j."""
+    k, v = _c(k_cache, np.uint16), _c(v_cache, np.uint16)
+    cu, ck, sel = _c(cu_seqlens, np.int32), _c(cu_k, np.int32), _c(sel_idx, np.int32)
+    L, T, Hkv, d = k.shape
+    B = cu.shape[0] - 1
+    Ktot = int(ck[-1])
+    assert v.shape == k.shape and sel.shape == (L, Hkv, Ktot)
+    pk = np.zeros((L, Ktot * Hkv, d), dtype=np.uint16)
+    pv = np.zeros_like(pk)
+    rc = _load().sgo_pack_kv(L, B, Hkv, d, _p(cu), _p(k), _p(v), _i64(T * Hkv * d), _i64(Hkv * d), _i64(d),
+                             _p(sel), _p(ck), _p(pk), _p(pv))
+    if rc:
+        raise RuntimeError("sgo_pack_kv failed: %d" % rc)
+    return pk, pv
+
+
+def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu_seqlens, local_idx, cu_nloc,
+                       softmax_scale: float = 0.0):
+    """(out float32 [B][H_q][d], lse float32 [B][H_q]) of attention over packed rows ++ indexed local rows.
+
+    q uint16 [B][H_q][d]; packed_k/v uint16 [K_tot*H_kv][d]; local_k/v uint16 [T][H_kv][d];
+    local_idx int32 [H_kv][NL_tot].
+    """
+    q, pk, pv = _c(q, np.uint16), _c(packed_k, np.uint16), _c(packed_v, np.uint16)
+    lk, lv = _c(local_k, np.uint16), _c(local_v, np.uint16)
+    cu, ck, cl, li = _c(cu_seqlens, np.int32), _c(cu_k, np.int32), _c(cu_nloc, np.int32), _c(local_idx, np.int32)
+    B, Hq, d = q.shape
+    T, Hkv, d2 = lk.shape
+    assert d == d2 and li.shape == (Hkv, int(cl[-1])) and pk.shape == (int(ck[-1]) * Hkv, d)
+    out = np.zeros((B, Hq, d), dtype=np.float32)
+    lse = np.zeros((B, Hq), dtype=np.float32)
+    rc = _load().sgo_sparse_decode_attn(B, Hq, Hkv, d, _p(cu), _p(q), _p(pk), _p(pv), _p(ck), _p(lk), _p(lv),
+                                        _i64(Hkv * d), _i64(d), _p(li), _p(cl), ctypes.c_double(softmax_scale),
+                                        _p(out), _p(lse))
+    if rc:
+        raise RuntimeError("sgo_sparse_decode_attn failed: %d" % rc)
+    return out, lse
+
+
+def split_index(kv_index, kv_mask, cu_seqlens, cu_k, reorder: bool = True):
+    """Algorithm 1.  Returns (reordered, local_index, remote_index, n_local [B][H_kv], n_remote [B][H_kv])."""
+    idx, mask = _c(kv_index, np.int32), _c(kv_mask, np.int8)
+    cu, ck = _c(cu_seqlens, np.int32), _c(cu_k, np.int32)
+    Hkv, Ktot = idx.shape
+    B = cu.shape[0] - 1
+    assert Ktot == ck[-1] and mask.shape == (int(cu[-1]),)
+    reordered = np.zeros_like(idx)
+    loc = np.full_like(idx, -1)
+    rem = np.full_like(idx, -1)
+    nl = np.zeros((B, Hkv), dtype=np.int32)
+    nr = np.zeros((B, Hkv), dtype=np.int32)
+    rc = _load().sgo_split_index(B, Hkv, _p(cu), _p(ck), _p(idx), _p(mask), int(bool(reorder)),
+                                 _p(reordered), _p(loc), _p(rem), _p(nl), _p(nr))
+    if rc:
+        raise RuntimeError("sgo_split_index failed: %d" % rc)
+    return reordered, loc, rem, nl, nr

@@ -1,0 +1,326 @@
+/*
+ * CPU oracle for the selective-KV hot path (TEST INFRASTRUCTURE, not a product path).
+ *
+ * Plain, slow, scalar C written from the paper's definitions.  It shares no code with the
+ * CUDA library and must never be called from it: only the tests, the smoke check and the
+ * benchmark's cpu-baseline leg load this file.
+ *
+ * Arithmetic: bf16 inputs are widened exactly; every dot product, exponential and sum is in
+ * double; results are rounded once to float.  The only parallelism is an OpenMP loop over
+ * independent (layer, sequence, KV head) units.
+ *
+ * Notation (paper, Section 2.1 / 2.3): H x N x d tensors per layer, attention
+ * softmax(Q K^T / sqrt(d)) V per head; the "KV index" is a BH x k matrix whose rows hold the k
+ * selected entries of one head of one request; the "selected KV" has shape BH x k x d.
+ * Here the batch is ragged: sequence b owns tokens cu[b] .. cu[b+1]-1 of a token-major cache.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int sgo_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void sgo_set_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/*
+ * Importance of every prompt token for every (layer, KV head).
+ *
+ * Section 4.1 defines a KV entry's importance through how often the selection algorithm picks
+ * it, and notes that all such algorithms rank entries by attention-score magnitude; S(e) in
+ * Eq. 1 is a plain count (a sum over occurrences).  The prefill side cannot see decode queries,
+ * so the last W prompt queries stand in for them: importance[t] is the attention mass
+ * (Section 2.1: softmax(q K^T / sqrt(d)), each query attending to itself and all previous
+ * tokens) that those W queries of the G query heads sharing KV head g put on token t, summed
+ * over the G*W rows without normalisation.
+ *
+ * q_win      bf16 [L][B][W][Hq][d]; row i of sequence b is the query at position N_b - W_eff + i,
+ *            W_eff = min(W, N_b); rows i >= W_eff are ignored.
+ * k_cache    bf16, element (l, token, g, c) at l*ls + token*ts + g*hs + c.
+ * importance float [L][Hkv][T].
+ */
+int sgo_score(int L, int B, int Hq, int Hkv, int d, int W, const int32_t *cu,
+              const uint16_t *q_win, const uint16_t *k_cache, int64_t ls, int64_t ts, int64_t hs,
+              float *importance) {
+    if (Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || W <= 0) return 1;
+    const int G = Hq / Hkv;
+    const int64_t T = cu[B];
+    const double inv_sqrt_d = 1.0 / sqrt((double)d);
+    int fail = 0;
+#pragma omp parallel for collapse(3) schedule(dynamic, 1)
+    for (int l = 0; l < L; ++l)
+        for (int b = 0; b < B; ++b)
+            for (int g = 0; g < Hkv; ++g) {
+                const int64_t c0 = cu[b];
+                const int N = cu[b + 1] - cu[b];
+                float *imp = importance + ((int64_t)l * Hkv + g) * T + c0;
+                if (N <= 0) continue;
+                const int Weff = W < N ? W : N;
+                double *acc = (double *)calloc((size_t)N, sizeof(double));
+                double *s = (double *)malloc((size_t)N * sizeof(double));
+                double *qd = (double *)malloc((size_t)d * sizeof(double));
+                if (!acc || !s || !qd) { fail = 1; free(acc); free(s); free(qd); continue; }
+                for (int hh = 0; hh < G; ++hh)
+                    for (int i = 0; i < Weff; ++i) {
+                        const int h = g * G + hh;
+                        const int pos = N - Weff + i;            /* position of this query in the prompt */
+                        const uint16_t *q = q_win + ((((int64_t)l * B + b) * W + i) * Hq + h) * d;
+                        for (int c = 0; c < d; ++c) qd[c] = bf16_to_double(q[c]);
+                        double mx = -INFINITY;
+                        for (int t = 0; t <= pos; ++t) {         /* causal: keys 0..pos are visible */
+                            const uint16_t *k = k_cache + l * ls + (c0 + t) * ts + g * hs;
+                            double dot = 0.0;
+                            for (int c = 0; c < d; ++c) dot += qd[c] * bf16_to_double(k[c]);
+                            s[t] = dot * inv_sqrt_d;
+                            if (s[t] > mx) mx = s[t];
+                        }
+                        double sum = 0.0;
+                        for (int t = 0; t <= pos; ++t) { s[t] = exp(s[t] - mx); sum += s[t]; }
+                        for (int t = 0; t <= pos; ++t) acc[t] += s[t] / sum;
+                    }
+                for (int t = 0; t < N; ++t) imp[t] = (float)acc[t];
+                free(acc); free(s); free(qd);
+            }
+    return fail;
+}
+
+/* Order-preserving image of a float's bit pattern: larger float <=> larger unsigned key.
+ * (+0 > -0; +inf above every finite value; NaNs ordered by their bit patterns.) */
+static uint32_t order_key(float x) {
+    uint32_t u;
+    memcpy(&u, &x, sizeof u);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+typedef struct { uint32_t key; int32_t t; } sgo_pair;
+
+static int cmp_key_desc_index_asc(const void *a, const void *b) {
+    const sgo_pair *x = (const sgo_pair *)a, *y = (const sgo_pair *)b;
+    if (x->key != y->key) return x->key > y->key ? -1 : 1;
+    return (x->t > y->t) - (x->t < y->t);
+}
+
+static int cmp_int_asc(const void *a, const void *b) {
+    const int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+/*
+ * Per-head top-k KV index (Section 2.3: each row of the BH x k KV index holds the top-k entries
+ * of one head of one request).  For (l, b, g) the k_b = cu_k[b+1]-cu_k[b] positions with the
+ * largest importance are kept; equal values go to the lower position; the row is emitted in
+ * ascending position order (entry order does not change attention, Section 4.2).
+ *
+ * importance float [L][Hkv][T];  sel_idx int32 [L][Hkv][K_tot], sequence-local positions.
+ * Returns 2 if some k_b is outside [0, N_b].
+ */
+int sgo_select_topk(int L, int B, int Hkv, const int32_t *cu, const float *importance,
+                    const int32_t *cu_k, int32_t *sel_idx) {
+    const int64_t T = cu[B], K_tot = cu_k[B];
+    for (int b = 0; b < B; ++b) {
+        const int kb = cu_k[b + 1] - cu_k[b];
+        if (kb < 0 || kb > cu[b + 1] - cu[b]) return 2;
+    }
+    int fail = 0;
+#pragma omp parallel for collapse(3) schedule(dynamic, 1)
+    for (int l = 0; l < L; ++l)
+        for (int b = 0; b < B; ++b)
+            for (int g = 0; g < Hkv; ++g) {
+                const int N = cu[b + 1] - cu[b];
+                const int kb = cu_k[b + 1] - cu_k[b];
+                if (kb == 0) continue;
+                const float *imp = importance + ((int64_t)l * Hkv + g) * T + cu[b];
+                int32_t *out = sel_idx + ((int64_t)l * Hkv + g) * K_tot + cu_k[b];
+                sgo_pair *p = (sgo_pair *)malloc((size_t)N * sizeof(sgo_pair));
+                if (!p) { fail = 1; continue; }
+                for (int t = 0; t < N; ++t) { p[t].key = order_key(imp[t]); p[t].t = t; }
+                qsort(p, (size_t)N, sizeof(sgo_pair), cmp_key_desc_index_asc);
+                for (int j = 0; j < kb; ++j) out[j] = p[j].t;
+                qsort(out, (size_t)kb, sizeof(int32_t), cmp_int_asc);
+                free(p);
+            }
+    return fail;
+}
+
+/*
+ * Gather-pack of the selected K/V rows into a contiguous buffer (Section 4.2: the selected KV
+ * has shape BH x k x d, a "row" being the k entries of one head; the prefill node "selects the
+ * required KV entries locally" before sending them).
+ *
+ * packed_k/v bf16 [L][K_tot*Hkv][d]; row of (b, g, j) is cu_k[b]*Hkv + g*k_b + j.
+ * Returns 3 if an index is outside its sequence.
+ */
+int sgo_pack_kv(int L, int B, int Hkv, int d, const int32_t *cu, const uint16_t *k_cache,
+                const uint16_t *v_cache, int64_t ls, int64_t ts, int64_t hs, const int32_t *sel_idx,
+                const int32_t *cu_k, uint16_t *packed_k, uint16_t *packed_v) {
+    const int64_t K_tot = cu_k[B];
+    int bad = 0;
+    for (int l = 0; l < L; ++l)
+        for (int b = 0; b < B; ++b)
+            for (int g = 0; g < Hkv; ++g) {
+                const int N = cu[b + 1] - cu[b];
+                const int kb = cu_k[b + 1] - cu_k[b];
+                for (int j = 0; j < kb; ++j) {
+                    const int32_t t = sel_idx[((int64_t)l * Hkv + g) * K_tot + cu_k[b] + j];
+                    if (t < 0 || t >= N) { bad = 3; continue; }
+                    const int64_t src = l * ls + ((int64_t)cu[b] + t) * ts + g * hs;
+                    const int64_t dst = (((int64_t)l * K_tot + cu_k[b]) * Hkv + (int64_t)g * kb + j) * d;
+                    memcpy(packed_k + dst, k_cache + src, (size_t)d * sizeof(uint16_t));
+                    memcpy(packed_v + dst, v_cache + src, (size_t)d * sizeof(uint16_t));
+                }
+            }
+    return bad;
+}
+
+/*
+ * Decode attention of one new query per (sequence, query head) over a two-source KV list
+ * (Section 4.2, two-lane fetching: the entries of a head arrive partly as contiguous rows at
+ * the start of its row of the selected KV, partly by gathering with a local index).  Since the
+ * order of KV entries along the sequence axis does not change softmax(q K^T / sqrt(d)) V, the
+ * result is plain attention over the concatenated list
+ *     [packed rows 0..k_b-1 of (b, g)] ++ [local rows cu[b] + local_idx[g][cu_nloc[b] + j]],
+ * computed here in one pass.  The list is a multiset: nothing is de-duplicated.
+ *
+ * q bf16 [B][Hq][d]; packed_k/v bf16 [K_tot*Hkv][d] (one layer, layout of sgo_pack_kv);
+ * local_k/v bf16, element (token, g, c) at token*ts + g*hs + c; local_idx int32 [Hkv][NL_tot].
+ * out float [B][Hq][d] (not rounded to bf16); lse float [B][Hq] = max + ln(sum).
+ * An empty list gives out = 0 and lse = -inf.  Returns 3 on an out-of-range local index.
+ */
+int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, const uint16_t *q,
+                           const uint16_t *packed_k, const uint16_t *packed_v, const int32_t *cu_k,
+                           const uint16_t *local_k, const uint16_t *local_v, int64_t ts, int64_t hs,
+                           const int32_t *local_idx, const int32_t *cu_nloc, double softmax_scale,
+                           float *out, float *lse) {
+    if (Hkv <= 0 || Hq % Hkv != 0) return 1;
+    const int G = Hq / Hkv;
+    const int64_t NL_tot = cu_nloc[B];
+    const double scale = softmax_scale > 0.0 ? softmax_scale : 1.0 / sqrt((double)d);
+    int bad = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hq; ++h) {
+            const int g = h / G;
+            const int N = cu[b + 1] - cu[b];
+            const int kb = cu_k[b + 1] - cu_k[b];
+            const int nl = cu_nloc[b + 1] - cu_nloc[b];
+            const int n = kb + nl;
+            float *o = out + ((int64_t)b * Hq + h) * d;
+            for (int c = 0; c < d; ++c) o[c] = 0.0f;
+            if (lse) lse[(int64_t)b * Hq + h] = -INFINITY;
+            if (n == 0) continue;
+            const uint16_t **kr = (const uint16_t **)malloc((size_t)n * sizeof(*kr));
+            const uint16_t **vr = (const uint16_t **)malloc((size_t)n * sizeof(*vr));
+            double *s = (double *)malloc((size_t)n * sizeof(double));
+            double *acc = (double *)calloc((size_t)d, sizeof(double));
+            int m = 0;
+            for (int j = 0; j < kb; ++j, ++m) {
+                const int64_t row = ((int64_t)cu_k[b] * Hkv + (int64_t)g * kb + j) * d;
+                kr[m] = packed_k + row;
+                vr[m] = packed_v + row;
+            }
+            for (int j = 0; j < nl; ++j) {
+                const int32_t t = local_idx[(int64_t)g * NL_tot + cu_nloc[b] + j];
+                if (t < 0 || t >= N) { bad = 3; continue; }
+                const int64_t off = ((int64_t)cu[b] + t) * ts + g * hs;
+                kr[m] = local_k + off;
+                vr[m] = local_v + off;
+                ++m;
+            }
+            const uint16_t *qq = q + ((int64_t)b * Hq + h) * d;
+            double mx = -INFINITY;
+            for (int j = 0; j < m; ++j) {
+                double dot = 0.0;
+                for (int c = 0; c < d; ++c) dot += bf16_to_double(qq[c]) * bf16_to_double(kr[j][c]);
+                s[j] = dot * scale;
+                if (s[j] > mx) mx = s[j];
+            }
+            double sum = 0.0;
+            for (int j = 0; j < m; ++j) { s[j] = exp(s[j] - mx); sum += s[j]; }
+            for (int j = 0; j < m; ++j)
+                for (int c = 0; c < d; ++c) acc[c] += s[j] * bf16_to_double(vr[j][c]);
+            if (m > 0) {
+                for (int c = 0; c < d; ++c) o[c] = (float)(acc[c] / sum);
+                if (lse) lse[(int64_t)b * Hq + h] = (float)(mx + log(sum));
+            }
+            free(kr); free(vr); free(s); free(acc);
+        }
+    return bad;
+}
+
+/*
+ * Algorithm 1 (KV index splitting and reordering), per row of the KV index.
+ *
+ *   (1) mask = kv_mask[kv_index]          -- one int8 per token, shared by all heads;
+ *                                            0 = padding, 1 = local, 2 = remote
+ *   (4,5) optional: sort each row of mask in descending order and apply the same order to
+ *         kv_index, so that remote entries (value 2) are contiguous at the start of the row;
+ *         the sort is stable, i.e. entries keep their original relative order in each class
+ *   (2) local_index  = kv_index[mask == 1]
+ *   (3) remote_index = kv_index[mask == 2]
+ *
+ * kv_index int32 [Hkv][K_tot] with prefix sums cu_k (sequence-local positions, row segment of
+ * (b, g) at g*K_tot + cu_k[b]); kv_mask int8 [T] ragged by cu.
+ * Outputs: reordered int32 [Hkv][K_tot] (the row after steps 4-5, or a copy when reorder == 0);
+ * local_index / remote_index int32 [Hkv][K_tot], each row segment filled from its start;
+ * n_local / n_remote int32 [B][Hkv].  Entries with mask 0 are dropped from both lists.
+ */
+int sgo_split_index(int B, int Hkv, const int32_t *cu, const int32_t *cu_k, const int32_t *kv_index,
+                    const int8_t *kv_mask, int reorder, int32_t *reordered, int32_t *local_index,
+                    int32_t *remote_index, int32_t *n_local, int32_t *n_remote) {
+    const int64_t K_tot = cu_k[B];
+    int bad = 0;
+    for (int b = 0; b < B; ++b)
+        for (int g = 0; g < Hkv; ++g) {
+            const int N = cu[b + 1] - cu[b];
+            const int kb = cu_k[b + 1] - cu_k[b];
+            const int64_t base = (int64_t)g * K_tot + cu_k[b];
+            int8_t *mask = (int8_t *)malloc((size_t)(kb > 0 ? kb : 1));
+            int32_t *row = (int32_t *)malloc((size_t)(kb > 0 ? kb : 1) * sizeof(int32_t));
+            for (int j = 0; j < kb; ++j) {
+                const int32_t t = kv_index[base + j];
+                row[j] = t;
+                if (t < 0 || t >= N) { bad = 3; mask[j] = 0; } else mask[j] = kv_mask[cu[b] + t];
+            }
+            if (reorder) {           /* stable descending sort of (mask, index) by mask: insertion sort */
+                for (int j = 1; j < kb; ++j) {
+                    const int8_t mj = mask[j];
+                    const int32_t rj = row[j];
+                    int i = j - 1;
+                    while (i >= 0 && mask[i] < mj) { mask[i + 1] = mask[i]; row[i + 1] = row[i]; --i; }
+                    mask[i + 1] = mj; row[i + 1] = rj;
+                }
+            }
+            int nl = 0, nr = 0;
+            for (int j = 0; j < kb; ++j) {
+                reordered[base + j] = row[j];
+                if (mask[j] == 1) local_index[base + nl++] = row[j];
+                else if (mask[j] == 2) remote_index[base + nr++] = row[j];
+            }
+            n_local[b * Hkv + g] = nl;
+            n_remote[b * Hkv + g] = nr;
+            free(mask); free(row);
+        }
+    return bad;
+}

@@ -1,0 +1,71 @@
+"""Pins for the oracle's Algorithm 1 (KV index splitting and reordering, Section 4.2)."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from helpers import cu_of
+
+
+def make(seed, lens=(30, 12), ks=(10, 12), Hkv=3, p=(0.1, 0.5, 0.4)):
+    rng = np.random.default_rng(seed)
+    cu, ck = cu_of(lens), cu_of(ks)
+    mask = rng.choice(np.array([0, 1, 2], dtype=np.int8), size=int(cu[-1]), p=p)
+    idx = np.zeros((Hkv, int(ck[-1])), dtype=np.int32)
+    for g in range(Hkv):
+        for b, n in enumerate(lens):
+            idx[g, ck[b]:ck[b + 1]] = np.sort(rng.choice(n, ks[b], replace=False))
+    return idx, mask, cu, ck
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_split_matches_numpy_indexing(seed):
+    """Operators 1-5 written with numpy fancy indexing and a library stable sort."""
+    idx, mask, cu, ck = make(seed)
+    re, loc, rem, nl, nr = oracle.split_index(idx, mask, cu, ck, reorder=True)
+    for g in range(idx.shape[0]):
+        for b in range(len(cu) - 1):
+            row = idx[g, ck[b]:ck[b + 1]]
+            m = mask[cu[b] + row]                                   # (1)
+            order = np.argsort(-m.astype(np.int32), kind="stable")  # (4)
+            row2, m2 = row[order], m[order]                         # (5)
+            assert re[g, ck[b]:ck[b + 1]].tolist() == row2.tolist()
+            assert loc[g, ck[b]: ck[b] + nl[b, g]].tolist() == row2[m2 == 1].tolist()   # (2)
+            assert rem[g, ck[b]: ck[b] + nr[b, g]].tolist() == row2[m2 == 2].tolist()   # (3)
+
+
+def test_split_partition_and_remote_first():
+    idx, mask, cu, ck = make(9, p=(0.0, 0.6, 0.4))
+    re, loc, rem, nl, nr = oracle.split_index(idx, mask, cu, ck, reorder=True)
+    for g in range(idx.shape[0]):
+        for b in range(len(cu) - 1):
+            row = set(idx[g, ck[b]:ck[b + 1]].tolist())
+            l = loc[g, ck[b]: ck[b] + nl[b, g]].tolist()
+            r = rem[g, ck[b]: ck[b] + nr[b, g]].tolist()
+            assert set(l) | set(r) == row and not (set(l) & set(r))          # no padding here: a partition
+            # descending mask order: the remote entries are the first n_remote entries of the reordered row
+            assert re[g, ck[b]: ck[b] + nr[b, g]].tolist() == r
+            assert re[g, ck[b] + nr[b, g]: ck[b + 1]].tolist() == l
+
+
+def test_split_without_reordering_keeps_row_order_and_drops_padding():
+    idx, mask, cu, ck = make(5)
+    re, loc, rem, nl, nr = oracle.split_index(idx, mask, cu, ck, reorder=False)
+    assert np.array_equal(re, idx)
+    for g in range(idx.shape[0]):
+        for b in range(len(cu) - 1):
+            row = idx[g, ck[b]:ck[b + 1]]
+            m = mask[cu[b] + row]
+            assert nl[b, g] + nr[b, g] == int((m != 0).sum())
+            assert loc[g, ck[b]: ck[b] + nl[b, g]].tolist() == row[m == 1].tolist()
+            assert rem[g, ck[b]: ck[b] + nr[b, g]].tolist() == row[m == 2].tolist()
+
+
+def test_mask_footprint_matches_printed_example():
+    path = os.path.join(os.path.dirname(__file__), "golden", "kv_mask_footprint.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    tokens, layers, per_layer, total_mb = int(rows[0][0]), int(rows[0][1]), int(rows[0][2]), float(rows[0][3])
+    mask = np.zeros(tokens, dtype=np.int8)            # the mask the oracle indexes: one int8 per token
+    assert mask.nbytes == per_layer == 64 * 1024
+    assert layers * mask.nbytes / 2**20 == total_mb
