@@ -1,0 +1,161 @@
+/*
+ * smartgen.h -- C ABI of the selective-KV hot path on one B200 (sm_100a).
+ *
+ * Four calls cover the path: on the prefill side, score every prompt token's importance for each
+ * (layer, KV head), pick each head's top-k tokens under a KV budget, and gather-pack the selected
+ * K/V rows into one contiguous transfer-ready buffer; on the decode side, attention whose keys and
+ * values come partly from that packed buffer and partly from an index-addressed local cache.
+ *
+ * Conventions shared by every call
+ *   - Every pointer named in a signature is a DEVICE pointer unless the comment says "host".
+ *     All device pointers must be 16-byte aligned.  The caller owns every buffer; the library
+ *     allocates nothing, keeps no state between calls and never synchronises the stream.
+ *   - bf16 tensors are passed as `const void*` / `void*` (raw bfloat16 bit patterns).
+ *   - The batch is ragged: sequence b owns tokens cu_seqlens[b] .. cu_seqlens[b+1]-1 of a
+ *     token-major cache; N_b = cu_seqlens[b+1] - cu_seqlens[b].
+ *   - The return value reports errors the host can see before launching (bad arguments,
+ *     unsupported shape, workspace too small, a failed CUDA call).  Problems only the device can
+ *     see (an index outside its sequence, a budget above the prompt length, a bounded wait that
+ *     expired) are OR-ed into *dev_status as (1 << sg_status) bits, if dev_status is not NULL,
+ *     and the offending row is skipped or clamped -- never dereferenced.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Inputs are never modified.  Calls are thread-safe given distinct streams and workspaces.
+ */
+#ifndef SMARTGEN_H_
+#define SMARTGEN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SG_OK = 0,
+  SG_ERR_INVALID = 1,     /* null or misaligned pointer, bad shape, k_b > N_b (device bit) ...   */
+  SG_ERR_UNSUPPORTED = 2, /* head_dim not 64/128, H_q % H_kv != 0, G*W beyond the built tiles ... */
+  SG_ERR_WORKSPACE = 3,   /* workspace_bytes < sg_workspace_bytes(...)                            */
+  SG_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see sg_last_cuda_error()          */
+  SG_ERR_INDEX = 5,       /* device bit: an index outside its sequence was skipped                */
+  SG_ERR_TIMEOUT = 6      /* device bit: a bounded wait inside a kernel expired                   */
+} sg_status;
+
+/* Operation ids for sg_workspace_bytes. */
+enum { SG_OP_SCORE = 0, SG_OP_SELECT_TOPK = 1, SG_OP_PACK_KV = 2, SG_OP_SPARSE_DECODE_ATTN = 3,
+       SG_OP_SPLIT_INDEX = 4 };
+
+/* Shape of one call (host memory, passed by const pointer).  Strides are in ELEMENTS (bf16). */
+typedef struct {
+  int32_t num_layers;         /* layers covered by this call (>= 1); decode/split: must be 1      */
+  int32_t batch;              /* B >= 1                                                           */
+  int32_t num_q_heads;        /* H_q                                                              */
+  int32_t num_kv_heads;       /* H_kv, H_q % H_kv == 0, G = H_q / H_kv <= 16                      */
+  int32_t head_dim;           /* d in {64, 128}                                                   */
+  int32_t window;             /* W, scoring window (sg_score only)                                */
+  int32_t total_tokens;       /* T = cu_seqlens[B]                                                */
+  int32_t max_seqlen;         /* an upper bound on every N_b (launch geometry, shared memory)     */
+  const int32_t* cu_seqlens;  /* device, B+1 ascending prefix sums, cu_seqlens[0] = 0             */
+  int64_t cache_layer_stride; /* elements between layers of the K (and V) cache                   */
+  int64_t cache_token_stride; /* elements between tokens  (H_kv*d when dense, multiple of 8)      */
+  int64_t cache_head_stride;  /* elements between KV heads (d when token-major, multiple of 8)    */
+} sg_shape;
+
+/* Bytes of device workspace the given operation needs for this shape.  total_sel = K_tot (sum of
+ * the per-sequence budgets k_b), total_loc = NL_tot (sum of the per-sequence local-index counts);
+ * pass 0 where an operation does not use them.  Returns 0 for operations that need none. */
+size_t sg_workspace_bytes(int op, const sg_shape* shape, int32_t total_sel, int32_t total_loc);
+
+/*
+ * sg_score -- importance of every prompt token for every (layer, KV head).
+ *
+ * Defines: the paper ranks KV entries by attention-score magnitude and counts how often an entry
+ * is picked (Section 4.1, definition of importance; S(e) in Eq. 1 is a sum over occurrences);
+ * attention is softmax(Q K^T / sqrt(d)) with each query seeing itself and all previous tokens
+ * (Section 2.1).  The last W prompt queries stand in for the decode queries the prefill side
+ * cannot see:
+ *     importance[l][g][cu[b]+t] = sum over the G query heads h of KV head g and the
+ *         W_eff = min(W, N_b) window rows i of softmax_t( q_{h,i} . k_{g,t} / sqrt(d) ),
+ *     the softmax of row i running over the keys t <= N_b - W_eff + i (its own position).
+ *
+ * q_win       bf16 [L][B][W][H_q][d], dense; row i of sequence b is the query at N_b - W_eff + i.
+ * k_cache     bf16, element (l, token, g, c) at l*layer_stride + token*token_stride + g*head_stride + c.
+ * importance  fp32 [L][H_kv][T], fully overwritten.
+ * Supported: G*W <= 512 and a multiple of 16 (d = 128) or <= 1024 (d = 64).
+ */
+sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
+                   void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+
+/*
+ * sg_select_topk -- per-head top-k KV index under a budget.
+ *
+ * Defines: a KV index row holds the k entries selected for one head of one request
+ * (Section 2.3, BH x k KV index).  For every (l, b, g) the k_b = cu_k[b+1] - cu_k[b] positions
+ * of sequence b with the largest importance are kept.  Order of values: the total order of the
+ * fp32 bit patterns (+0 above -0, +inf above every finite value -- so entries given infinite
+ * importance as in Eq. 1 are always kept); equal values go to the lower position.  Each row is
+ * emitted in ascending position order (entry order does not change attention, Section 4.2).
+ *
+ * importance  fp32 [L][H_kv][T].
+ * cu_k        device int32 [B+1], prefix sums of k_b; total_sel = cu_k[B] (host copy of the total).
+ * sel_idx     int32 [L][H_kv][K_tot]; the row segment of (l, g, b) starts at cu_k[b]; positions
+ *             are sequence-local (0 .. N_b-1).  k_b > N_b sets the SG_ERR_INVALID device bit and
+ *             the row is filled with 0 .. N_b-1 followed by -1.
+ */
+sg_status sg_select_topk(const sg_shape* shape, const float* importance, const int32_t* cu_k,
+                         int32_t total_sel, int32_t* sel_idx, void* workspace, size_t workspace_bytes,
+                         int32_t* dev_status, void* stream);
+
+/*
+ * sg_pack_kv -- gather the selected K/V rows into a contiguous, transfer-ready buffer.
+ *
+ * Defines: the selected KV has shape BH x k x d, a "row" being the k entries of one head
+ * (Section 4.2); the prefill node selects the required entries locally before sending them.
+ *     packed_k[l][cu_k[b]*H_kv + g*k_b + j][:] = k_cache[l][cu[b] + sel_idx[l][g][cu_k[b]+j]][g][:]
+ * and the same for V.  An index outside [0, N_b) sets the SG_ERR_INDEX device bit and its row is
+ * written as zeros.
+ *
+ * packed_k/v  bf16 [L][K_tot*H_kv][d], fully overwritten.
+ */
+sg_status sg_pack_kv(const sg_shape* shape, const void* k_cache, const void* v_cache,
+                     const int32_t* sel_idx, const int32_t* cu_k, int32_t total_sel, void* packed_k,
+                     void* packed_v, int32_t* dev_status, void* stream);
+
+/*
+ * sg_sparse_decode_attn -- one decode step of attention over a two-source KV list.
+ *
+ * Defines: two-lane KV fetching (Section 4.2): the entries a head needs arrive partly as
+ * contiguous rows at the start of its row of the selected KV (the packed buffer) and partly by
+ * gathering with a local index from the decode node's own cache.  Because the order of KV
+ * entries along the sequence axis does not change softmax(q K^T / sqrt(d)) V (Section 4.2), the
+ * result for (b, h), g = h / G, is plain attention (Section 2.1) over the multiset
+ *     [packed rows 0..k_b-1 of (b, g)] ++ [local rows cu[b] + local_idx[g][cu_nloc[b]+j], j < n_loc_b],
+ * computed as split-softmax partials merged through their log-sum-exps.  Nothing is
+ * de-duplicated.  A local index outside [0, N_b) sets the SG_ERR_INDEX device bit and is skipped.
+ *
+ * shape       num_layers must be 1; cache strides describe local_k / local_v.
+ * q           bf16 [B][H_q][d].
+ * packed_k/v  bf16 [K_tot*H_kv][d], layout of sg_pack_kv for one layer; cu_k as in sg_pack_kv.
+ * local_k/v   bf16, element (token, g, c) at token*token_stride + g*head_stride + c.
+ * local_idx   int32 [H_kv][NL_tot]; cu_nloc device int32 [B+1]; total_loc = cu_nloc[B].
+ * softmax_scale  0 means 1/sqrt(d).
+ * out         bf16 [B][H_q][d]; lse fp32 [B][H_q] (may be NULL) = max + ln(sum) of the scaled
+ *             scores.  A head with an empty list gets out = 0 and lse = -inf.
+ */
+sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void* packed_k,
+                                const void* packed_v, const int32_t* cu_k, int32_t total_sel,
+                                const void* local_k, const void* local_v, const int32_t* local_idx,
+                                const int32_t* cu_nloc, int32_t total_loc, float softmax_scale,
+                                void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                int32_t* dev_status, void* stream);
+
+/* Static description of a status code. */
+const char* sg_strerror(sg_status status);
+
+/* cudaError_t (or CUresult for driver calls) of the last failed CUDA call on this host thread. */
+int sg_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SMARTGEN_H_ */

@@ -1,0 +1,188 @@
+"""ctypes binding of libsmartgen.so: same names as the C ABI, argument marshalling only.
+
+Every function takes torch CUDA tensors (PyTorch is used for device memory and streams, nothing
+else), checks dtypes/contiguity, passes raw pointers to the library and raises `SmartGenError` on a
+non-zero status.  All computation happens in the library's CUDA kernels; there is no fallback --
+importing this module without the built library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsmartgen.so")
+
+SG_OK, SG_ERR_INVALID, SG_ERR_UNSUPPORTED, SG_ERR_WORKSPACE, SG_ERR_CUDA, SG_ERR_INDEX, SG_ERR_TIMEOUT = range(7)
+SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_SPLIT_INDEX = range(5)
+
+# every symbol include/smartgen.h declares
+EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
+            "sg_strerror", "sg_last_cuda_error")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libsmartgen.so is not built (%s): run `python __graft_entry__.py` or "
+                      "`python -m paper_2607_28150_b200.build`; there is no CPU fallback" % LIB_PATH)
+_lib = ctypes.CDLL(LIB_PATH)
+
+
+class SmartGenError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.sg_strerror(status).decode()
+        if status == SG_ERR_CUDA:
+            msg += " [cuda error %d]" % _lib.sg_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg))
+
+
+class Shape(ctypes.Structure):
+    """Mirror of `sg_shape`."""
+    _fields_ = [("num_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+                ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("window", ctypes.c_int32),
+                ("total_tokens", ctypes.c_int32), ("max_seqlen", ctypes.c_int32),
+                ("cu_seqlens", ctypes.c_void_p), ("cache_layer_stride", ctypes.c_int64),
+                ("cache_token_stride", ctypes.c_int64), ("cache_head_stride", ctypes.c_int64)]
+
+
+_vp, _i32, _sz, _f = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t, ctypes.c_float
+_sp = ctypes.POINTER(Shape)
+_lib.sg_strerror.restype = ctypes.c_char_p
+_lib.sg_strerror.argtypes = [ctypes.c_int]
+_lib.sg_last_cuda_error.restype = ctypes.c_int
+_lib.sg_workspace_bytes.restype = _sz
+_lib.sg_workspace_bytes.argtypes = [ctypes.c_int, _sp, _i32, _i32]
+_lib.sg_score.restype = ctypes.c_int
+_lib.sg_score.argtypes = [_sp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.sg_select_topk.restype = ctypes.c_int
+_lib.sg_select_topk.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _sz, _vp, _vp]
+_lib.sg_pack_kv.restype = ctypes.c_int
+_lib.sg_pack_kv.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
+_lib.sg_sparse_decode_attn.restype = ctypes.c_int
+_lib.sg_sparse_decode_attn.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp,
+                                       _sz, _vp, _vp]
+
+
+def make_shape(num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
+               cu_seqlens: torch.Tensor, total_tokens: int, max_seqlen: int,
+               layer_stride: Optional[int] = None, token_stride: Optional[int] = None,
+               head_stride: Optional[int] = None) -> Shape:
+    """Build an `sg_shape`.  `cu_seqlens` is a device int32 tensor of B+1 prefix sums; the caller passes the
+    host-side totals (no device read happens here).  Strides default to a dense [L][T][H_kv][d] cache."""
+    _check(cu_seqlens, torch.int32, "cu_seqlens")
+    ts = num_kv_heads * head_dim if token_stride is None else token_stride
+    hs = head_dim if head_stride is None else head_stride
+    ls = total_tokens * ts if layer_stride is None else layer_stride
+    s = Shape(num_layers, cu_seqlens.numel() - 1, num_q_heads, num_kv_heads, head_dim, window, total_tokens,
+              max_seqlen, cu_seqlens.data_ptr(), ls, ts, hs)
+    s._keep = cu_seqlens          # keep the device array alive as long as the struct
+    return s
+
+
+def _check(t: Optional[torch.Tensor], dtype, name: str, allow_none: bool = False):
+    if t is None:
+        if allow_none:
+            return
+        raise TypeError("%s is required" % name)
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    dtypes = dtype if isinstance(dtype, (tuple, list)) else (dtype,)
+    if t.dtype not in dtypes:
+        raise TypeError("%s: expected dtype %s, got %s" % (name, dtypes, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous (strided caches go through the sg_shape strides)" % name)
+
+
+_BF16 = (torch.bfloat16, torch.int16, torch.uint16)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    return getattr(stream, "cuda_stream", stream) or None
+
+
+def _ws(workspace: Optional[torch.Tensor]):
+    if workspace is None:
+        return None, 0
+    return workspace.data_ptr(), workspace.numel() * workspace.element_size()
+
+
+def sg_strerror(status: int) -> str:
+    return _lib.sg_strerror(status).decode()
+
+
+def sg_last_cuda_error() -> int:
+    return int(_lib.sg_last_cuda_error())
+
+
+def sg_workspace_bytes(op: int, shape: Shape, total_sel: int = 0, total_loc: int = 0) -> int:
+    return int(_lib.sg_workspace_bytes(op, ctypes.byref(shape), total_sel, total_loc))
+
+
+def alloc_workspace(op: int, shape: Shape, total_sel: int = 0, total_loc: int = 0, device="cuda") -> Optional[torch.Tensor]:
+    """Device scratch of the size the library asks for (None when the operation needs none)."""
+    n = sg_workspace_bytes(op, shape, total_sel, total_loc)
+    return torch.empty(n, dtype=torch.uint8, device=device) if n else None
+
+
+def sg_score(shape: Shape, q_win: torch.Tensor, k_cache: torch.Tensor, importance: torch.Tensor,
+             workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(q_win, _BF16, "q_win"); _check(k_cache, _BF16, "k_cache"); _check(importance, torch.float32, "importance")
+    _check(dev_status, torch.int32, "dev_status", True)
+    w, wb = _ws(workspace)
+    rc = _lib.sg_score(ctypes.byref(shape), _ptr(q_win), k_cache.data_ptr(), _ptr(importance), w, wb,
+                       _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_score")
+
+
+def sg_select_topk(shape: Shape, importance: torch.Tensor, cu_k: torch.Tensor, total_sel: int,
+                   sel_idx: torch.Tensor, workspace: Optional[torch.Tensor] = None,
+                   dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(importance, torch.float32, "importance"); _check(cu_k, torch.int32, "cu_k")
+    _check(sel_idx, torch.int32, "sel_idx"); _check(dev_status, torch.int32, "dev_status", True)
+    w, wb = _ws(workspace)
+    rc = _lib.sg_select_topk(ctypes.byref(shape), _ptr(importance), cu_k.data_ptr(), total_sel, _ptr(sel_idx), w, wb,
+                             _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_select_topk")
+
+
+def sg_pack_kv(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tensor, sel_idx: torch.Tensor,
+               cu_k: torch.Tensor, total_sel: int, packed_k: torch.Tensor, packed_v: torch.Tensor,
+               dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(k_cache, _BF16, "k_cache"); _check(v_cache, _BF16, "v_cache"); _check(sel_idx, torch.int32, "sel_idx")
+    _check(cu_k, torch.int32, "cu_k"); _check(packed_k, _BF16, "packed_k"); _check(packed_v, _BF16, "packed_v")
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_pack_kv(ctypes.byref(shape), k_cache.data_ptr(), v_cache.data_ptr(), _ptr(sel_idx), cu_k.data_ptr(),
+                         total_sel, _ptr(packed_k), _ptr(packed_v), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_pack_kv")
+
+
+def sg_sparse_decode_attn(shape: Shape, q: torch.Tensor, packed_k: Optional[torch.Tensor],
+                          packed_v: Optional[torch.Tensor], cu_k: torch.Tensor, total_sel: int,
+                          local_k: Optional[torch.Tensor], local_v: Optional[torch.Tensor],
+                          local_idx: Optional[torch.Tensor], cu_nloc: torch.Tensor, total_loc: int,
+                          out: torch.Tensor, lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                          workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                          stream=None) -> None:
+    _check(q, _BF16, "q"); _check(out, _BF16, "out"); _check(cu_k, torch.int32, "cu_k")
+    _check(cu_nloc, torch.int32, "cu_nloc"); _check(packed_k, _BF16, "packed_k", True)
+    _check(packed_v, _BF16, "packed_v", True); _check(local_k, _BF16, "local_k", True)
+    _check(local_v, _BF16, "local_v", True); _check(local_idx, torch.int32, "local_idx", True)
+    _check(lse, torch.float32, "lse", True); _check(dev_status, torch.int32, "dev_status", True)
+    w, wb = _ws(workspace)
+    rc = _lib.sg_sparse_decode_attn(ctypes.byref(shape), q.data_ptr(), _ptr(packed_k), _ptr(packed_v), cu_k.data_ptr(),
+                                    total_sel, _ptr(local_k), _ptr(local_v), _ptr(local_idx), cu_nloc.data_ptr(),
+                                    total_loc, softmax_scale, out.data_ptr(), _ptr(lse), w, wb, _ptr(dev_status),
+                                    _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_sparse_decode_attn")

@@ -1,0 +1,484 @@
+// sg_sparse_decode_attn: split-KV decode attention over a packed source plus an index-gathered source.
+//
+// Memory-bound: every attended token costs 2*d*2 bytes of K+V per KV head and only 4*G*d flops.
+// The token list of a (sequence, KV head) -- packed rows first, then local rows addressed through
+// local_idx -- is cut into chunks; one CTA streams one chunk through a 3-stage cp.async ring of
+// 64-token K/V tiles in shared memory (16-byte copies, XOR-swizzled rows so ldmatrix is
+// conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).
+// Each warp owns 16 tokens of a tile: S = Q K^T and O += P V run on bf16 tensor-core MMAs with the
+// G query rows of the KV head padded to 16, the online softmax (base 2) stays in registers.
+// Per-chunk partials (m, l, unnormalised O) go to the workspace; a second kernel merges them with
+// the log-sum-exp rule and writes bf16 out and fp32 lse.
+#include "common.cuh"
+#include "launch.h"
+
+namespace sg {
+namespace {
+
+constexpr int kDecThreads = 128;
+constexpr int kDecWarps = 4;
+constexpr int kTile = 64;          // tokens per pipeline stage
+constexpr int kStages = 3;
+constexpr int kMaxChunk = 2048;    // tokens per work item (index staging buffer)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct DecParams {
+  const uint16_t* q;
+  const uint16_t* packed_k;
+  const uint16_t* packed_v;
+  const uint16_t* local_k;
+  const uint16_t* local_v;
+  const int32_t* cu;
+  const int32_t* cu_k;
+  const int32_t* cu_nloc;
+  const int32_t* local_idx;
+  float* part_o;     // [max_items][Hkv][G][D]   unnormalised
+  float* part_ml;    // [max_items][Hkv][G][2]   (m in log2 units, l)
+  uint16_t* out;
+  float* lse;
+  int32_t* dev_status;
+  int64_t ts, hs;
+  int32_t B, Hq, Hkv, G, K_tot, NL_tot, chunk;
+  float scale_log2;
+};
+
+// Work item -> (sequence b, chunk c within b, first item of b).  Computed redundantly per warp.
+__device__ __forceinline__ bool find_item(const DecParams& p, int item, int lane, int& b_out, int& c_out) {
+  int acc = 0;
+  for (int b0 = 0; b0 < p.B; b0 += 32) {
+    const int b = b0 + lane;
+    int nch = 0;
+    if (b < p.B) {
+      const int n = (p.cu_k[b + 1] - p.cu_k[b]) + (p.cu_nloc[b + 1] - p.cu_nloc[b]);
+      nch = (n + p.chunk - 1) / p.chunk;
+    }
+    int inc = nch;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, off);
+      if (lane >= off) inc += v;
+    }
+    const int tot = __shfl_sync(0xffffffffu, inc, 31);
+    if (item < acc + tot) {
+      const unsigned hit = __ballot_sync(0xffffffffu, item < acc + inc);
+      const int src = __ffs(hit) - 1;
+      const int exc = __shfl_sync(0xffffffffu, inc - nch, src);
+      b_out = b0 + src;
+      c_out = item - (acc + exc);
+      return true;
+    }
+    acc += tot;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// kHi: the KV head has more than 8 query rows, so MMA rows 8..15 carry data too.
+template <int D, bool kHi>
+__global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const DecParams p) {
+  constexpr int kRowBytes = D * 2;
+  constexpr int kChunksPerRow = D / 8;                       // 16-byte chunks
+  constexpr int kTileBytes = kTile * kRowBytes;
+  constexpr int kCopiesPerThread = kTile * kChunksPerRow / kDecThreads;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  uint8_t* sk = smem_raw;                                    // [kStages][kTile][D] bf16, swizzled
+  uint8_t* sv = smem_raw + kStages * kTileBytes;
+  int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw + 2 * kStages * kTileBytes);   // [kMaxChunk]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = blockIdx.y;
+  int b, c;
+  if (!find_item(p, blockIdx.x, lane, b, c)) return;
+  const int kb = p.cu_k[b + 1] - p.cu_k[b];
+  const int nl = p.cu_nloc[b + 1] - p.cu_nloc[b];
+  const int c0 = p.cu[b];
+  const int nseq = p.cu[b + 1] - c0;
+  const int pos_beg = c * p.chunk;
+  const int pos_end = min(kb + nl, pos_beg + p.chunk);
+  const int ntok = pos_end - pos_beg;
+  const int ntiles = (ntok + kTile - 1) / kTile;
+
+  // Stage this chunk's local indices (validated); packed positions get 0.
+  for (int i = tid; i < ntok; i += kDecThreads) {
+    const int pos = pos_beg + i;
+    int v = 0;
+    if (pos >= kb) {
+      v = __ldg(p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + (pos - kb));
+      if (v < 0 || v >= nseq) { v = -1; raise(p.dev_status, SG_ERR_INDEX); }
+    }
+    s_idx[i] = v;
+  }
+  __syncthreads();
+
+  const uint16_t* pk_base = p.packed_k + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
+  const uint16_t* pv_base = p.packed_v + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
+  const uint16_t* lk_base = p.local_k + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
+  const uint16_t* lv_base = p.local_v + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
+  const uint32_t sk_u32 = smem_u32(sk), sv_u32 = smem_u32(sv);
+
+  auto load_tile = [&](int tile, int stage) {
+#pragma unroll
+    for (int i = 0; i < kCopiesPerThread; ++i) {
+      const int qid = tid + i * kDecThreads;
+      const int row = qid / kChunksPerRow;
+      const int col = qid % kChunksPerRow;
+      const int li = tile * kTile + row;                      // index within the chunk
+      const int pos = pos_beg + li;
+      const uint16_t* srck = p.packed_k;
+      const uint16_t* srcv = p.packed_v;
+      int bytes = 0;
+      if (li < ntok) {
+        if (pos < kb) {
+          srck = pk_base + (int64_t)pos * D + col * 8;
+          srcv = pv_base + (int64_t)pos * D + col * 8;
+          bytes = 16;
+        } else {
+          const int t = s_idx[li];
+          if (t >= 0) {
+            srck = lk_base + (int64_t)t * p.ts + col * 8;
+            srcv = lv_base + (int64_t)t * p.ts + col * 8;
+            bytes = 16;
+          }
+        }
+      }
+      const uint32_t off = stage * kTileBytes + row * kRowBytes + ((col ^ (row & 7)) << 4);
+      cp_async16(sk_u32 + off, srck, bytes);
+      cp_async16(sv_u32 + off, srcv, bytes);
+    }
+  };
+
+  // Q fragments (A operand, 16 x D, rows >= G are zero).
+  const int r_lo = lane >> 2, r_hi = r_lo + 8;
+  uint32_t qa[D / 16][4];
+  {
+    const uint16_t* qb = p.q + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+      const int col = kk * 16 + 2 * (lane & 3);
+      qa[kk][0] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col) : 0u;
+      qa[kk][2] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col + 8) : 0u;
+      qa[kk][1] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col) : 0u;
+      qa[kk][3] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col + 8) : 0u;
+    }
+  }
+
+  float o_acc[D / 8][4];
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+
+#pragma unroll
+  for (int s = 0; s < kStages - 1; ++s) {
+    if (s < ntiles) load_tile(s, s);
+    cp_async_commit();
+  }
+
+#pragma unroll 1
+  for (int tile = 0; tile < ntiles; ++tile) {
+    cp_async_wait<kStages - 2>();
+    __syncthreads();
+    {
+      const int nt = tile + kStages - 1;
+      if (nt < ntiles) load_tile(nt, nt % kStages);
+      cp_async_commit();
+    }
+    const int stage = tile % kStages;
+    const uint32_t k_st = sk_u32 + stage * kTileBytes;
+    const uint32_t v_st = sv_u32 + stage * kTileBytes;
+    const int wrow = warp * 16;
+    if (tile * kTile + wrow >= ntok) continue;               // this warp's 16 tokens are all padding
+
+    // S = Q K^T for 16 tokens (two n8 tiles)
+    float s_acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    {
+      const int mi = lane >> 3;
+      const int row = wrow + (mi >> 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const int chunk = kk * 2 + (mi & 1);
+        uint32_t kf[4];
+        ldmatrix_x4(kf, k_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+        mma_bf16(s_acc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[0], kf[1]);
+        mma_bf16(s_acc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[2], kf[3]);
+      }
+    }
+    // online softmax in base 2; mask padding and skipped indices
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int li = tile * kTile + wrow + j * 8 + 2 * (lane & 3) + e;
+        const bool valid = li < ntok && s_idx[li] >= 0;
+        s_acc[j][e] = valid ? s_acc[j][e] * p.scale_log2 : -INFINITY;
+        mx_lo = fmaxf(mx_lo, s_acc[j][e]);
+        if (kHi) {
+          s_acc[j][2 + e] = valid ? s_acc[j][2 + e] * p.scale_log2 : -INFINITY;
+          mx_hi = fmaxf(mx_hi, s_acc[j][2 + e]);
+        }
+      }
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo);
+    const float mu_lo = mn_lo == -INFINITY ? 0.f : mn_lo;
+    const float al_lo = exp2f(m_lo - mu_lo);
+    m_lo = mn_lo;
+    float mu_hi = 0.f, al_hi = 1.f;
+    if (kHi) {
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+      const float mn_hi = fmaxf(m_hi, mx_hi);
+      mu_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+      al_hi = exp2f(m_hi - mu_hi);
+      m_hi = mn_hi;
+    }
+    float sum_lo = 0.f, sum_hi = 0.f;
+    uint32_t pa[4];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float p0 = exp2f(s_acc[j][0] - mu_lo), p1 = exp2f(s_acc[j][1] - mu_lo);
+      sum_lo += p0 + p1;
+      pa[2 * j] = pack_bf16(p0, p1);
+      if (kHi) {
+        const float p2 = exp2f(s_acc[j][2] - mu_hi), p3 = exp2f(s_acc[j][3] - mu_hi);
+        sum_hi += p2 + p3;
+        pa[2 * j + 1] = pack_bf16(p2, p3);
+      } else {
+        pa[2 * j + 1] = 0u;
+      }
+    }
+    sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1);
+    sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
+    l_lo = l_lo * al_lo + sum_lo;
+    if (kHi) {
+      sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1);
+      sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
+      l_hi = l_hi * al_hi + sum_hi;
+    }
+    const bool rescale = kHi ? (al_lo != 1.f || al_hi != 1.f) : (al_lo != 1.f);
+    if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll
+      for (int i = 0; i < D / 8; ++i) {
+        o_acc[i][0] *= al_lo; o_acc[i][1] *= al_lo;
+        if (kHi) { o_acc[i][2] *= al_hi; o_acc[i][3] *= al_hi; }
+      }
+    }
+    // O += P V
+    {
+      const int mi = lane >> 3;
+      const int row = wrow + (mi & 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int dc = 0; dc < D / 16; ++dc) {
+        const int chunk = dc * 2 + (mi >> 1);
+        uint32_t vf[4];
+        ldmatrix_x4_trans(vf, v_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+        mma_bf16(o_acc[2 * dc], pa[0], pa[1], pa[2], pa[3], vf[0], vf[1]);
+        mma_bf16(o_acc[2 * dc + 1], pa[0], pa[1], pa[2], pa[3], vf[2], vf[3]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+
+  // merge the four warps through shared memory (the pipeline buffers are free now)
+  float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
+  float* sm_m = sm_o + kDecWarps * 16 * D;                    // [kDecWarps][16]
+  float* sm_l = sm_m + kDecWarps * 16;
+  if ((lane & 3) == 0) {
+    sm_m[warp * 16 + r_lo] = m_lo; sm_l[warp * 16 + r_lo] = l_lo;
+    sm_m[warp * 16 + r_hi] = kHi ? m_hi : -INFINITY; sm_l[warp * 16 + r_hi] = kHi ? l_hi : 0.f;
+  }
+#pragma unroll
+  for (int i = 0; i < D / 8; ++i) {
+    const int col = i * 8 + 2 * (lane & 3);
+    float* dst = sm_o + (warp * 16 + r_lo) * D + col;
+    dst[0] = o_acc[i][0]; dst[1] = o_acc[i][1];
+    if (kHi) { dst[8 * D] = o_acc[i][2]; dst[8 * D + 1] = o_acc[i][3]; }
+  }
+  __syncthreads();
+  const int64_t slot = (int64_t)blockIdx.x * p.Hkv + g;
+  float* po = p.part_o + slot * p.G * D;
+  float* pml = p.part_ml + slot * p.G * 2;
+  for (int e = tid; e < p.G * D; e += kDecThreads) {
+    const int r = e / D, col = e - r * D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, sm_m[w * 16 + r]);
+    const float Mu = M == -INFINITY ? 0.f : M;
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+      const float f = exp2f(sm_m[w * 16 + r] - Mu);
+      L += sm_l[w * 16 + r] * f;
+      O += sm_o[(w * 16 + r) * D + col] * f;
+    }
+    po[e] = O;
+    if (col == 0) { pml[2 * r] = M; pml[2 * r + 1] = L; }
+  }
+}
+
+// Merge the per-chunk partials of one (sequence, query head): m = max m_j, l = sum l_j 2^(m_j-m),
+// o = sum o_j 2^(m_j-m) / l.  One block of D threads per (h, b).
+template <int D>
+__global__ void __launch_bounds__(D) decode_combine_kernel(const DecParams p) {
+  __shared__ int s_part[D / 32];
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int g = h / p.G, r = h - g * p.G;
+  // first work item of sequence b = number of chunks of the sequences before it
+  int cnt = 0;
+  for (int bb = tid; bb < b; bb += D) {
+    const int n = (p.cu_k[bb + 1] - p.cu_k[bb]) + (p.cu_nloc[bb + 1] - p.cu_nloc[bb]);
+    cnt += (n + p.chunk - 1) / p.chunk;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+  if ((tid & 31) == 0) s_part[tid >> 5] = cnt;
+  __syncthreads();
+  int first = 0;
+#pragma unroll
+  for (int w = 0; w < D / 32; ++w) first += s_part[w];
+  const int n = (p.cu_k[b + 1] - p.cu_k[b]) + (p.cu_nloc[b + 1] - p.cu_nloc[b]);
+  const int nch = (n + p.chunk - 1) / p.chunk;
+
+  float M = -INFINITY;
+  for (int c = 0; c < nch; ++c) M = fmaxf(M, p.part_ml[(((int64_t)(first + c) * p.Hkv + g) * p.G + r) * 2]);
+  const float Mu = M == -INFINITY ? 0.f : M;
+  float L = 0.f, O = 0.f;
+  for (int c = 0; c < nch; ++c) {
+    const int64_t slot = (int64_t)(first + c) * p.Hkv + g;
+    const float f = exp2f(p.part_ml[(slot * p.G + r) * 2] - Mu);
+    L += p.part_ml[(slot * p.G + r) * 2 + 1] * f;
+    O += p.part_o[(slot * p.G + r) * D + tid] * f;
+  }
+  const float res = L > 0.f ? O / L : 0.f;
+  reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.Hq + h) * D + tid] = __float2bfloat16_rn(res);
+  if (p.lse && tid == 0) p.lse[(int64_t)b * p.Hq + h] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+}
+
+template <int D>
+constexpr int decode_smem_bytes() { return 2 * kStages * kTile * D * 2 + kMaxChunk * 4; }
+
+}  // namespace
+
+int decode_chunk_tokens(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
+  const int64_t total = (int64_t)total_sel + total_loc;
+  const int target_items = (4 * kNumSMs + shape->num_kv_heads - 1) / shape->num_kv_heads;   // ~4 CTAs per SM
+  int64_t chunk = (total + target_items - 1) / target_items;
+  chunk = ((chunk + kTile - 1) / kTile) * kTile;
+  if (chunk < kTile) chunk = kTile;
+  if (chunk > kMaxChunk) chunk = kMaxChunk;
+  return (int)chunk;
+}
+
+static int64_t decode_max_items(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
+  const int chunk = decode_chunk_tokens(shape, total_sel, total_loc);
+  return ((int64_t)total_sel + total_loc + chunk - 1) / chunk + shape->batch;
+}
+
+size_t decode_workspace_bytes(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
+  if (shape->num_kv_heads < 1 || shape->num_q_heads < 1) return 0;
+  const int64_t items = decode_max_items(shape, total_sel, total_loc);
+  const int G = shape->num_q_heads / shape->num_kv_heads;
+  return (size_t)items * shape->num_kv_heads * G * (shape->head_dim + 2) * sizeof(float);
+}
+
+}  // namespace sg
+
+extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void* packed_k,
+                                           const void* packed_v, const int32_t* cu_k, int32_t total_sel,
+                                           const void* local_k, const void* local_v, const int32_t* local_idx,
+                                           const int32_t* cu_nloc, int32_t total_loc, float softmax_scale,
+                                           void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                           int32_t* dev_status, void* stream) {
+  using namespace sg;
+  sg_status st = check_shape(shape, false);
+  if (st != SG_OK) return st;
+  if (shape->num_layers != 1 || total_sel < 0 || total_loc < 0) return SG_ERR_INVALID;
+  if (!q || !out || !cu_k || !cu_nloc) return SG_ERR_INVALID;
+  if (total_sel > 0 && (!packed_k || !packed_v)) return SG_ERR_INVALID;
+  if (total_loc > 0 && (!local_k || !local_v || !local_idx)) return SG_ERR_INVALID;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(cu_k) || !aligned16(cu_nloc) || !aligned16(packed_k) ||
+      !aligned16(packed_v) || !aligned16(local_k) || !aligned16(local_v) || !aligned16(local_idx) ||
+      !aligned16(workspace) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
+    return SG_ERR_INVALID;
+  if (!(softmax_scale >= 0.f)) return SG_ERR_INVALID;
+  const size_t need = decode_workspace_bytes(shape, total_sel, total_loc);
+  if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
+
+  const int D = shape->head_dim;
+  const int G = shape->num_q_heads / shape->num_kv_heads;
+  const int64_t items = decode_max_items(shape, total_sel, total_loc);
+  if (items > 0x7fffffffLL || shape->num_kv_heads > 65535 || shape->batch > 65535) return SG_ERR_UNSUPPORTED;
+  DecParams p;
+  p.q = static_cast<const uint16_t*>(q);
+  p.packed_k = static_cast<const uint16_t*>(packed_k ? packed_k : q);
+  p.packed_v = static_cast<const uint16_t*>(packed_v ? packed_v : q);
+  p.local_k = static_cast<const uint16_t*>(local_k ? local_k : q);
+  p.local_v = static_cast<const uint16_t*>(local_v ? local_v : q);
+  p.cu = shape->cu_seqlens;
+  p.cu_k = cu_k;
+  p.cu_nloc = cu_nloc;
+  p.local_idx = local_idx;
+  p.part_o = static_cast<float*>(workspace);
+  p.part_ml = p.part_o + items * shape->num_kv_heads * G * D;
+  p.out = static_cast<uint16_t*>(out);
+  p.lse = lse;
+  p.dev_status = dev_status;
+  p.ts = shape->cache_token_stride;
+  p.hs = shape->cache_head_stride;
+  p.B = shape->batch;
+  p.Hq = shape->num_q_heads;
+  p.Hkv = shape->num_kv_heads;
+  p.G = G;
+  p.K_tot = total_sel;
+  p.NL_tot = total_loc;
+  p.chunk = decode_chunk_tokens(shape, total_sel, total_loc);
+  p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const dim3 grid1((unsigned)items, (unsigned)shape->num_kv_heads);
+  const dim3 grid2((unsigned)shape->num_q_heads, (unsigned)shape->batch);
+#define SG_LAUNCH_DECODE(DD, HI)                                                                                \
+  do {                                                                                                          \
+    SG_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<DD, HI>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                     decode_smem_bytes<DD>()));                                                 \
+    decode_partial_kernel<DD, HI><<<grid1, kDecThreads, decode_smem_bytes<DD>(), s>>>(p);                        \
+  } while (0)
+  if (total_sel + total_loc > 0) {
+    if (D == 128) { if (G > 8) SG_LAUNCH_DECODE(128, true); else SG_LAUNCH_DECODE(128, false); }
+    else          { if (G > 8) SG_LAUNCH_DECODE(64, true);  else SG_LAUNCH_DECODE(64, false); }
+    SG_CUDA_TRY(cudaGetLastError());
+  }
+#undef SG_LAUNCH_DECODE
+  if (D == 128) decode_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
+  else decode_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
+  SG_CUDA_TRY(cudaGetLastError());
+  return SG_OK;
+}

@@ -1,0 +1,201 @@
+// sg_select_topk: per-(layer, sequence, KV head) top-k by MSB-first radix select.
+//
+// One CTA owns one importance row.  The row's fp32 values are mapped to order-preserving uint32
+// keys and kept in shared memory (rows of up to ~55K tokens; longer rows are re-read from L2).
+// Four 8-bit histogram passes find the k-th largest key exactly; a final ordered compaction
+// (ballot + prefix counts, no atomics) emits the selected positions in ascending order, taking
+// equal-to-threshold entries from the lowest positions first.  The result is therefore a pure
+// function of the input row: identical on every run and identical to a full sort.
+#include "common.cuh"
+
+namespace sg {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kHistCopies = 8;
+constexpr int kMaxSmemBytes = 227 * 1024;
+constexpr int kSelFixedSmem = (kHistCopies * 256 + 256 + 4 * kSelWarps + 8) * 4;
+constexpr int kSelKeyCap = (kMaxSmemBytes - kSelFixedSmem) / 4;
+
+struct SelParams {
+  const float* importance;
+  const int32_t* cu;
+  const int32_t* cu_k;
+  int32_t* sel_idx;
+  int32_t* dev_status;
+  int64_t T;
+  int32_t K_tot, B, Hkv;
+};
+
+// Takes the raw bit pattern: the row is read as uint32 so that no float instruction (and no
+// flush-to-zero of subnormals) ever touches the values.
+__device__ __forceinline__ uint32_t order_key(uint32_t u) {
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <bool kInSmem>
+__global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelParams p) {
+  extern __shared__ __align__(16) uint32_t smem[];
+  uint32_t* hist = smem;                              // [kHistCopies][256]
+  uint32_t* total = hist + kHistCopies * 256;         // [256]
+  uint32_t* wgt = total + 256;                        // [kSelWarps] per-warp counts / bases
+  uint32_t* weq = wgt + kSelWarps;
+  uint32_t* wgt_base = weq + kSelWarps;
+  uint32_t* weq_base = wgt_base + kSelWarps;
+  uint32_t* sh = weq_base + kSelWarps;                // [0] chosen bin, [1] remaining need
+  uint32_t* keys = sh + 8;                            // [N] when kInSmem
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = blockIdx.x;
+  const int l = row / (p.B * p.Hkv);
+  const int rem = row - l * (p.B * p.Hkv);
+  const int b = rem / p.Hkv;
+  const int g = rem - b * p.Hkv;
+  const int c0 = p.cu[b];
+  const int N = p.cu[b + 1] - c0;
+  const int ck = p.cu_k[b];
+  const int kb = p.cu_k[b + 1] - ck;
+  if (kb <= 0) return;
+  int32_t* out = p.sel_idx + ((int64_t)l * p.Hkv + g) * p.K_tot + ck;
+  if (kb >= N) {                                      // whole prompt (or an over-sized budget)
+    if (kb > N && tid == 0) raise(p.dev_status, SG_ERR_INVALID);
+    for (int j = tid; j < kb; j += kSelThreads) out[j] = j < N ? j : -1;
+    return;
+  }
+  const uint32_t* x = reinterpret_cast<const uint32_t*>(p.importance) + ((int64_t)l * p.Hkv + g) * p.T + c0;
+
+  if (kInSmem) {
+    for (int t = tid; t < N; t += kSelThreads) keys[t] = order_key(__ldg(x + t));
+  }
+  auto key_at = [&](int t) -> uint32_t { return kInSmem ? keys[t] : order_key(__ldg(x + t)); };
+
+  // ---- radix select: find the kb-th largest key ----
+  uint32_t prefix = 0, decided = 0, need = (uint32_t)kb;
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = tid; i < kHistCopies * 256; i += kSelThreads) hist[i] = 0;
+    __syncthreads();
+    uint32_t* my_hist = hist + (warp % kHistCopies) * 256;
+    for (int t = tid; t < N; t += kSelThreads) {
+      const uint32_t k = key_at(t);
+      if ((k & decided) == prefix) atomicAdd(&my_hist[(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t s = 0;
+#pragma unroll
+      for (int c = 0; c < kHistCopies; ++c) s += hist[c * 256 + tid];
+      total[tid] = s;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t c[8], s = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = total[255 - (lane * 8 + i)]; s += c[i]; }
+      uint32_t inc = s;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += v;
+      }
+      const uint32_t exc = inc - s;                   // candidates in bins above this lane's bins
+      if (exc < need && need <= inc) {
+        uint32_t run = exc;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (run < need && need <= run + c[i]) { sh[0] = 255u - (uint32_t)(lane * 8 + i); sh[1] = need - run; }
+          run += c[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= sh[0] << shift;
+    decided |= 255u << shift;
+    need = sh[1];
+    __syncthreads();
+  }
+  const uint32_t tau = prefix;                        // the kb-th largest key
+  const uint32_t need_eq = need;                      // entries equal to tau to keep, lowest positions first
+
+  // ---- ordered compaction: warp w owns positions [w*C, (w+1)*C) ----
+  const int C = (((N + kSelWarps - 1) / kSelWarps) + 31) & ~31;
+  const int beg = warp * C;
+  const int end = min(N, beg + C);
+  uint32_t ngt = 0, neq = 0;
+  for (int t0 = beg; t0 < end; t0 += 32) {
+    const int t = t0 + lane;
+    const uint32_t k = t < end ? key_at(t) : 0u;
+    ngt += __popc(__ballot_sync(0xffffffffu, t < end && k > tau));
+    neq += __popc(__ballot_sync(0xffffffffu, t < end && k == tau));
+  }
+  if (lane == 0) { wgt[warp] = ngt; weq[warp] = neq; }
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t a = wgt[lane], e = weq[lane], ia = a, ie = e;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t va = __shfl_up_sync(0xffffffffu, ia, off);
+      const uint32_t ve = __shfl_up_sync(0xffffffffu, ie, off);
+      if (lane >= off) { ia += va; ie += ve; }
+    }
+    wgt_base[lane] = ia - a;
+    weq_base[lane] = ie - e;
+  }
+  __syncthreads();
+  uint32_t gt_run = wgt_base[warp], eq_run = weq_base[warp];
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (int t0 = beg; t0 < end; t0 += 32) {
+    const int t = t0 + lane;
+    const uint32_t k = t < end ? key_at(t) : 0u;
+    const bool is_gt = t < end && k > tau;
+    const bool is_eq = t < end && k == tau;
+    const uint32_t bg = __ballot_sync(0xffffffffu, is_gt);
+    const uint32_t be = __ballot_sync(0xffffffffu, is_eq);
+    const uint32_t gt_before = gt_run + __popc(bg & lt_mask);
+    const uint32_t eq_before = eq_run + __popc(be & lt_mask);
+    if (is_gt || (is_eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = t;
+    gt_run += __popc(bg);
+    eq_run += __popc(be);
+  }
+}
+
+}  // namespace
+}  // namespace sg
+
+extern "C" sg_status sg_select_topk(const sg_shape* shape, const float* importance, const int32_t* cu_k,
+                                    int32_t total_sel, int32_t* sel_idx, void* workspace,
+                                    size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  using namespace sg;
+  (void)workspace;
+  (void)workspace_bytes;
+  sg_status st = check_shape(shape, false);
+  if (st != SG_OK) return st;
+  if (total_sel < 0) return SG_ERR_INVALID;
+  if (total_sel == 0) return SG_OK;
+  if (!importance || !cu_k || !sel_idx) return SG_ERR_INVALID;
+  if (!aligned16(importance) || !aligned16(cu_k) || !aligned16(sel_idx)) return SG_ERR_INVALID;
+  SelParams p;
+  p.importance = importance;
+  p.cu = shape->cu_seqlens;
+  p.cu_k = cu_k;
+  p.sel_idx = sel_idx;
+  p.dev_status = dev_status;
+  p.T = shape->total_tokens;
+  p.K_tot = total_sel;
+  p.B = shape->batch;
+  p.Hkv = shape->num_kv_heads;
+  const int64_t rows = (int64_t)shape->num_layers * shape->batch * shape->num_kv_heads;
+  if (rows > 0x7fffffffLL) return SG_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (shape->max_seqlen <= kSelKeyCap) {
+    const int smem = kSelFixedSmem + shape->max_seqlen * 4;
+    SG_CUDA_TRY(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    select_topk_kernel<true><<<(unsigned)rows, kSelThreads, smem, s>>>(p);
+  } else {
+    select_topk_kernel<false><<<(unsigned)rows, kSelThreads, kSelFixedSmem, s>>>(p);
+  }
+  SG_CUDA_TRY(cudaGetLastError());
+  return SG_OK;
+}

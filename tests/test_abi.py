@@ -1,0 +1,53 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares, and rejects bad
+arguments on the host before any launch."""
+import ctypes
+import os
+import re
+
+import paper_2607_28150_b200.binding as sg
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "smartgen.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sg_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    lib = ctypes.CDLL(sg.LIB_PATH)
+    names = declared_symbols()
+    assert set(sg.EXPORTED) <= set(names) and len(names) >= 7
+    for n in names:
+        assert hasattr(lib, n), n
+        assert hasattr(sg, n), "binding lacks %s" % n
+
+
+def test_strerror_covers_every_status():
+    msgs = [sg.sg_strerror(i) for i in range(7)]
+    assert msgs[0] == "ok" and len(set(msgs)) == 7
+
+
+def test_host_side_argument_checks_need_no_gpu():
+    lib = ctypes.CDLL(sg.LIB_PATH)
+    lib.sg_pack_kv.restype = ctypes.c_int
+    # null shape
+    assert lib.sg_pack_kv(None, None, None, None, None, 0, None, None, None, None) == sg.SG_ERR_INVALID
+    fake = ctypes.c_void_p(0x1000)
+    s = sg.Shape(1, 1, 8, 2, 96, 4, 16, 16, 0x1000, 16 * 2 * 96, 2 * 96, 96)
+    assert lib.sg_pack_kv(ctypes.byref(s), fake, fake, fake, fake, 4, fake, fake, None, None) == sg.SG_ERR_UNSUPPORTED
+    s = sg.Shape(1, 1, 8, 3, 128, 4, 16, 16, 0x1000, 16 * 3 * 128, 3 * 128, 128)
+    assert lib.sg_pack_kv(ctypes.byref(s), fake, fake, fake, fake, 4, fake, fake, None, None) == sg.SG_ERR_UNSUPPORTED
+    s = sg.Shape(1, 1, 8, 2, 128, 4, 16, 16, 0x1000, 16 * 256, 256, 128)
+    bad = ctypes.c_void_p(0x1004)        # misaligned
+    assert lib.sg_pack_kv(ctypes.byref(s), bad, fake, fake, fake, 4, fake, fake, None, None) == sg.SG_ERR_INVALID
+    assert lib.sg_pack_kv(ctypes.byref(s), fake, fake, fake, fake, -1, fake, fake, None, None) == sg.SG_ERR_INVALID
+    # decode: workspace too small is reported before any launch
+    lib.sg_sparse_decode_attn.restype = ctypes.c_int
+    lib.sg_sparse_decode_attn.argtypes = sg._lib.sg_sparse_decode_attn.argtypes
+    rc = lib.sg_sparse_decode_attn(ctypes.byref(s), fake, fake, fake, fake, 4, fake, fake, fake, fake, 4, 0.0, fake,
+                                   None, fake, 16, None, None)
+    assert rc == sg.SG_ERR_WORKSPACE
+    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 4, 4) > 16
+    assert sg.sg_workspace_bytes(sg.SG_OP_PACK_KV, s, 4, 4) == 0
