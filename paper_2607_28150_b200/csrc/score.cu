@@ -1,6 +1,605 @@
+// sg_score: window-query x key-cache scoring with a fused softmax and row-reduce (sm_100a).
+//
+// For one (layer, sequence, KV head) the R = G*W window queries are scored against all N keys:
+// a dense R x N x d contraction, so it runs on the 5th-generation tensor cores.  importance[t] =
+// sum_r softmax_row_r(s)[t] needs every row's normaliser before any probability can be summed
+// down a column, so the work is two passes over the keys:
+//
+//   pass 1 (row statistics)  D[row r][key t]  = Q_blk (A, 128 rows) x K_tile^T (B, 128 keys):
+//          each epilogue thread owns one query row (one TMEM lane) and keeps a running
+//          (max, sum-of-exp2) over the key columns -- no cross-thread reduction.
+//   pass 2 (column sums)     D[key t][row r]  = K_tile (A, 128 keys) x Q_blk^T (B, <=128 rows):
+//          each epilogue thread owns one key (one TMEM lane) and adds exp2(s*c - lse_r) over the
+//          query-row columns; lse_r is a per-column constant read from shared memory.
+//
+// Both passes share one warp-specialised skeleton: warp 0 feeds 128-key K tiles (and Q once) with
+// TMA into 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM
+// accumulator stages, warps 2-9 (two per TMEM lane quarter, each taking half of the columns)
+// drain them with tcgen05.ld.  The score matrix never leaves the SM.  Per-chunk row statistics
+// (pass 1) go to a small workspace; pass 2 merges them in its prologue.
+//
+// Every mbarrier wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word,
+// stops issuing work, drains its own TMA copies with bounded waits, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "common.cuh"
 #include "launch.h"
-namespace sg { size_t score_workspace_bytes(const sg_shape*) { return 0; } }
-extern "C" sg_status sg_score(const sg_shape*, const void*, const void*, float*, void*, size_t, int32_t*, void*) {
-  return SG_ERR_UNSUPPORTED;
+
+namespace sg {
+namespace {
+
+constexpr int kScoreThreads = 320;        // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-9: epilogue
+constexpr int kEpiThreads = 256;
+constexpr int kTileKeys = 128;
+constexpr int kAccStages = 4;             // 4 x 128 fp32 columns = the whole 512-column TMEM
+constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxKStages = 4;
+constexpr int kSmemLimit = 232448;        // 227 KB opt-in dynamic shared memory per CTA
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct ScoreParams {
+  const int32_t* cu;
+  float* importance;
+  float* part_m;           // [L][Hkv][max_items][Ralloc]
+  float* part_l;
+  int32_t* dev_status;
+  int64_t T;
+  int32_t B, Hkv, G, W, R, Rpad, Ralloc;
+  int32_t tiles_per_chunk, max_items, k_stages;
+  float scale_log2;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after about one second, or as soon as another thread has set *abort_flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    if (*abort_flag) return false;
+    if ((it & 255u) == 255u) {
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B): 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
+  d |= (uint64_t)(1024u >> 4) << 32;              // stride byte offset, bits [32,46)
+  d |= (uint64_t)1 << 46;                         // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                         // layout type: SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__device__ __forceinline__ uint32_t make_idesc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Work item -> (sequence, chunk of key tiles); also returns the sequence's first item.
+__device__ __forceinline__ bool find_chunk(const ScoreParams& p, int item, int lane, int& b_out, int& c_out, int& first_out, int& nch_out) {
+  int acc = 0;
+  for (int b0 = 0; b0 < p.B; b0 += 32) {
+    const int b = b0 + lane;
+    int nch = 0;
+    if (b < p.B) {
+      const int tiles = (p.cu[b + 1] - p.cu[b] + kTileKeys - 1) / kTileKeys;
+      nch = (tiles + p.tiles_per_chunk - 1) / p.tiles_per_chunk;
+    }
+    int inc = nch;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, inc, off);
+      if (lane >= off) inc += v;
+    }
+    const int tot = __shfl_sync(0xffffffffu, inc, 31);
+    if (item < acc + tot) {
+      const unsigned hit = __ballot_sync(0xffffffffu, item < acc + inc);
+      const int src = __ffs(hit) - 1;
+      const int exc = __shfl_sync(0xffffffffu, inc - nch, src);
+      b_out = b0 + src;
+      first_out = acc + exc;
+      c_out = item - first_out;
+      nch_out = __shfl_sync(0xffffffffu, nch, src);
+      return true;
+    }
+    acc += tot;
+  }
+  return false;
+}
+
+template <int D, bool kPass1>
+__global__ void __launch_bounds__(kScoreThreads, 1)
+score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
+  constexpr int kSub = D / 64;                        // 64-element (128-byte) sub-tiles along d
+  constexpr int kKSubBytes = kTileKeys * 128;         // one sub-tile of a K stage
+  constexpr int kKStageBytes = kSub * kKSubBytes;
+  extern __shared__ uint8_t smem_dyn[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  const int q_sub_bytes = p.Ralloc * 128;
+  uint8_t* q_smem = smem;
+  uint8_t* k_smem = q_smem + kSub * q_sub_bytes;
+  uint8_t* tail = k_smem + p.k_stages * kKStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 1 + 4*4 barriers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 17 * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 17 * 8 + 4);
+  float* sm_f = reinterpret_cast<float*>(tail + 160);         // pass 1: m[2][Ralloc], l[2][Ralloc]; pass 2: lse2[Ralloc], part[2][128]
+
+  const uint32_t bar_q = smem_u32(&bars[0]);
+  auto bar_kfull = [&](int s) { return smem_u32(&bars[1 + s]); };
+  auto bar_kempty = [&](int s) { return smem_u32(&bars[1 + kMaxKStages + s]); };
+  auto bar_afull = [&](int s) { return smem_u32(&bars[1 + 2 * kMaxKStages + s]); };
+  auto bar_aempty = [&](int s) { return smem_u32(&bars[1 + 2 * kMaxKStages + kAccStages + s]); };
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = blockIdx.y, l = blockIdx.z;
+  int b, chunk, first_item, nch;
+  if (!find_chunk(p, blockIdx.x, lane, b, chunk, first_item, nch)) return;
+  const int c0 = p.cu[b];
+  const int N = p.cu[b + 1] - c0;
+  const int Weff = min(p.W, N);
+  const int tiles_total = (N + kTileKeys - 1) / kTileKeys;
+  const int tile_beg = chunk * p.tiles_per_chunk;
+  const int tile_end = min(tiles_total, tile_beg + p.tiles_per_chunk);
+  const int nblk = kPass1 ? (p.R + 127) / 128 : (p.Rpad + 127) / 128;
+  const int first_win = N - Weff;                     // position of window row 0; keys <= it are visible to all rows
+
+  if (tid == 0) {
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < kMaxKStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
+    for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), kEpiThreads / 32); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish();
+  }
+  if (p.R < p.Ralloc) {
+    // Rows R..Ralloc-1 of the Q operand are never written by TMA: zero them so that padded MMA rows/columns
+    // are finite.  (The 128-byte swizzle only permutes 16-byte chunks inside a row's own 128 bytes.)
+    const int words = (p.Ralloc - p.R) * 32;
+    for (int dc = 0; dc < kSub; ++dc) {
+      uint32_t* z = reinterpret_cast<uint32_t*>(q_smem + dc * q_sub_bytes + p.R * 128);
+      for (int i = tid; i < words; i += kScoreThreads) z[i] = 0u;
+    }
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_arrive_expect_tx(bar_q, (uint32_t)(kSub * p.G * p.W * 128));
+#pragma unroll
+      for (int dc = 0; dc < kSub; ++dc)
+        tma_load_4d(smem_u32(q_smem + dc * q_sub_bytes), &tmap_q, bar_q, dc * 64, g * p.G, 0, l * p.B + b);
+      int stage = 0, issued = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
+        ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
+#pragma unroll
+        for (int dc = 0; dc < kSub; ++dc)
+          tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, g,
+                      c0 + tile * kTileKeys, l);
+        ++issued;
+        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
+      }
+      // Wait until the MMAs have released every stage: after this no arrival on a K barrier is pending.
+      for (int i = 0; i < p.k_stages && ok; ++i) {
+        ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
+        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        // Drain: wait (bounded) until every copy this thread issued has landed, so none is in flight at exit.
+        volatile int never = 0;
+        mbar_wait(bar_q, 0, &never);
+        for (int i = 0; i < issued; ++i) {
+          const int s = i % p.k_stages;
+          const uint32_t ph = (uint32_t)((i / p.k_stages) & 1);
+          if (i + p.k_stages >= issued) mbar_wait(bar_kfull(s), ph, &never);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      tc_fence_after();
+      int ks = 0, as = 0;
+      uint32_t kph = 0, aph = 0;
+      const uint32_t q_addr = smem_u32(q_smem);
+      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
+        ok = mbar_wait(bar_kfull(ks), kph, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
+        for (int blk = 0; blk < nblk && ok; ++blk) {
+          ok = mbar_wait(bar_aempty(as), aph ^ 1u, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int ncols = kPass1 ? 128 : min(128, p.Rpad - blk * 128);
+          const uint32_t idesc = make_idesc(128, ncols);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
+#pragma unroll
+          for (int dc = 0; dc < kSub; ++dc) {
+            const uint32_t qa = q_addr + dc * q_sub_bytes + blk * (128 * 128);
+            const uint32_t ka = k_addr + dc * kKSubBytes;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              const uint64_t dq = smem_desc_sw128(qa + kk * 32);
+              const uint64_t dk = smem_desc_sw128(ka + kk * 32);
+              umma_bf16(d_tmem, kPass1 ? dq : dk, kPass1 ? dk : dq, idesc, (dc | kk) != 0 ? 1u : 0u);
+            }
+          }
+          umma_commit(bar_afull(as));
+          if (++as == kAccStages) { as = 0; aph ^= 1u; }
+        }
+        if (ok) umma_commit(bar_kempty(ks));
+        if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int etid = tid - 64;
+    const int half = (warp - 2) >> 2;                  // which 64 accumulator columns this warp drains
+    const int lane_grp = warp & 3;                     // TMEM lane quarter this warp may access
+    const int row_in_tile = lane_grp * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+    const size_t part_base = (((size_t)l * p.Hkv + g) * p.max_items) * p.Ralloc;
+    int as = 0;
+    uint32_t aph = 0;
+    bool ok = true;
+
+    if (kPass1) {
+      float* sm_m = sm_f;                              // [2][Ralloc]
+      float* sm_l = sm_f + 2 * p.Ralloc;
+      for (int r = etid; r < 2 * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
+      epi_bar_sync();
+      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
+        const int t0 = tile * kTileKeys;
+        const bool all_visible = t0 + kTileKeys - 1 <= first_win;
+        for (int blk = 0; blk < nblk && ok; ++blk) {
+          ok = mbar_wait(bar_afull(as), aph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int r = blk * 128 + row_in_tile;
+          const bool row_ok = r < p.R && (r / p.G) < Weff;
+          const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
+          float m = sm_m[half * p.Ralloc + r], lsum = sm_l[half * p.Ralloc + r];
+#pragma unroll 1
+          for (int j = 0; j < 2; ++j) {
+            const int col0 = half * 64 + j * 32;
+            float v[32];
+            tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
+            if (all_visible && row_ok) {
+              float mx = v[0];
+#pragma unroll
+              for (int c = 1; c < 32; ++c) mx = fmaxf(mx, v[c]);
+              const float mn = fmaxf(m, mx * p.scale_log2);
+              float s = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) s += exp2f(fmaf(v[c], p.scale_log2, -mn));
+              lsum = lsum * exp2f(m - mn) + s;
+              m = mn;
+            } else if (col0 <= cmax) {
+              float mx = -INFINITY;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, v[c]) : mx;
+              const float mn = fmaxf(m, mx * p.scale_log2);
+              float s = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) s += (col0 + c <= cmax) ? exp2f(fmaf(v[c], p.scale_log2, -mn)) : 0.f;
+              lsum = lsum * exp2f(m - mn) + s;
+              m = mn;
+            }
+          }
+          sm_m[half * p.Ralloc + r] = m;
+          sm_l[half * p.Ralloc + r] = lsum;
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_aempty(as));
+          if (++as == kAccStages) { as = 0; aph ^= 1u; }
+        }
+      }
+      epi_bar_sync();
+      if (ok && !*abort_flag) {
+        const size_t slot = part_base + (size_t)blockIdx.x * p.Ralloc;
+        for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
+          const float m0 = sm_m[r], m1 = sm_m[p.Ralloc + r];
+          const float M = fmaxf(m0, m1);
+          const float Mu = M == -INFINITY ? 0.f : M;
+          p.part_m[slot + r] = M;
+          p.part_l[slot + r] = sm_l[r] * exp2f(m0 - Mu) + sm_l[p.Ralloc + r] * exp2f(m1 - Mu);
+        }
+      }
+    } else {
+      float* lse2 = sm_f;                              // [Ralloc]
+      float* sm_part = sm_f + p.Ralloc;                // [2][128]
+      for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
+        float val = INFINITY;                          // rows outside the window: exp2(x - inf) = 0
+        if (r < p.R && (r / p.G) < Weff) {
+          float M = -INFINITY;
+          for (int c = 0; c < nch; ++c) M = fmaxf(M, p.part_m[part_base + (size_t)(first_item + c) * p.Ralloc + r]);
+          float L = 0.f;
+          for (int c = 0; c < nch; ++c) {
+            const size_t o = part_base + (size_t)(first_item + c) * p.Ralloc + r;
+            L += p.part_l[o] * exp2f(p.part_m[o] - M);
+          }
+          val = M + log2f(L);
+        }
+        lse2[r] = val;
+      }
+      epi_bar_sync();
+      for (int tile = tile_beg; tile < tile_end; ++tile) {   // no early exit: every warp meets the named barrier
+        const int t = tile * kTileKeys + row_in_tile;  // this thread's key
+        const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
+        const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
+        float acc = 0.f;
+        for (int blk = 0; blk < nblk && ok; ++blk) {
+          ok = mbar_wait(bar_afull(as), aph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int ncols = min(128, p.Rpad - blk * 128);
+#pragma unroll 1
+          for (int j = 0; j < 2; ++j) {
+            const int col0 = half * 64 + j * 32;
+            if (col0 >= ncols) break;
+            float v[32];
+            tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
+            const float* ls = lse2 + blk * 128 + col0;
+            if (all_visible && col0 + 32 <= ncols) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                acc += exp2f(fmaf(v[c], p.scale_log2, -l4.x));
+                acc += exp2f(fmaf(v[c + 1], p.scale_log2, -l4.y));
+                acc += exp2f(fmaf(v[c + 2], p.scale_log2, -l4.z));
+                acc += exp2f(fmaf(v[c + 3], p.scale_log2, -l4.w));
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
+                acc += vis ? exp2f(fmaf(v[c], p.scale_log2, -ls[c])) : 0.f;
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_aempty(as));
+          if (++as == kAccStages) { as = 0; aph ^= 1u; }
+        }
+        float* part = sm_part + (tile & 1) * 128;
+        if (half == 1) part[row_in_tile] = acc;
+        epi_bar_sync();
+        if (half == 0 && ok && t < N)
+          p.importance[((size_t)l * p.Hkv + g) * p.T + c0 + t] = acc + part[row_in_tile];
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (tid == 0 && *abort_flag) raise(p.dev_status, SG_ERR_TIMEOUT);
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+    if (qres != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  }();
+  return fn;
+}
+
+struct ScorePlan {
+  int R, Rpad, Ralloc, k_stages, tiles_per_chunk, max_items, smem_bytes;
+  bool ok;
+};
+
+ScorePlan plan_score(const sg_shape* s) {
+  ScorePlan pl{};
+  const int D = s->head_dim;
+  const int G = s->num_q_heads / s->num_kv_heads;
+  pl.R = G * s->window;
+  pl.Rpad = (pl.R + 15) & ~15;
+  pl.Ralloc = (pl.R + 127) & ~127;
+  const int q_bytes = pl.Ralloc * D * 2;
+  const int k_stage = kTileKeys * D * 2;
+  const int tail = 160 + 4 * pl.Ralloc * 4 + 2 * 128 * 4;
+  const int avail = kSmemLimit - 1024 - q_bytes - tail;
+  pl.k_stages = avail / k_stage;
+  if (pl.k_stages > kMaxKStages) pl.k_stages = kMaxKStages;
+  pl.ok = pl.k_stages >= 2 && s->window <= 256 && pl.R <= 1024;
+  pl.smem_bytes = 1024 + q_bytes + pl.k_stages * k_stage + tail;
+  if (pl.smem_bytes < 120 * 1024) pl.smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes the whole TMEM
+  // chunking of the key axis: about four waves of CTAs over the SMs, 4..32 tiles per chunk
+  const int64_t total_tiles = ((int64_t)s->total_tokens / kTileKeys + s->batch) * s->num_kv_heads * s->num_layers;
+  int64_t tpc = total_tiles / (4 * kNumSMs);
+  if (tpc < 4) tpc = 4;
+  if (tpc > 32) tpc = 32;
+  pl.tiles_per_chunk = (int)tpc;
+  const int64_t max_tiles = (int64_t)s->total_tokens / kTileKeys + s->batch;
+  pl.max_items = (int)(max_tiles / pl.tiles_per_chunk + s->batch);
+  return pl;
+}
+
+}  // namespace
+
+size_t score_workspace_bytes(const sg_shape* s) {
+  if (s->num_kv_heads < 1 || s->num_q_heads < 1 || s->window < 1) return 0;
+  const ScorePlan pl = plan_score(s);
+  return (size_t)2 * s->num_layers * s->num_kv_heads * pl.max_items * pl.Ralloc * sizeof(float);
+}
+
+}  // namespace sg
+
+extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
+                              void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+  using namespace sg;
+  sg_status st = check_shape(shape, true);
+  if (st != SG_OK) return st;
+  if (shape->total_tokens == 0) return SG_OK;
+  if (!q_win || !k_cache || !importance) return SG_ERR_INVALID;
+  if (!aligned16(q_win) || !aligned16(k_cache) || !aligned16(importance) || !aligned16(workspace)) return SG_ERR_INVALID;
+  const ScorePlan pl = plan_score(shape);
+  if (!pl.ok) return SG_ERR_UNSUPPORTED;
+  if (shape->num_kv_heads > 65535 || shape->num_layers > 65535) return SG_ERR_UNSUPPORTED;
+  const size_t need = score_workspace_bytes(shape);
+  if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return cuda_fail((int)cudaErrorUnknown);
+
+  const int D = shape->head_dim;
+  const int G = shape->num_q_heads / shape->num_kv_heads;
+  CUtensorMap tmap_q, tmap_k;
+  {
+    // q_win [L*B][W][H_q][d]; box = (64 of d, G heads, W rows, 1) -> rows ordered (window row, head in group)
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)shape->num_q_heads, (cuuint64_t)shape->window,
+                                (cuuint64_t)shape->num_layers * shape->batch};
+    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)shape->num_q_heads * D * 2,
+                                   (cuuint64_t)shape->window * shape->num_q_heads * D * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)shape->window, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q_win), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail((int)r);
+  }
+  {
+    // k_cache viewed as (d, H_kv, T, L) with the caller's strides; box = 64 of d x 1 head x 128 tokens
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)shape->num_kv_heads, (cuuint64_t)shape->total_tokens,
+                                (cuuint64_t)shape->num_layers};
+    const cuuint64_t hs = shape->num_kv_heads > 1 ? (cuuint64_t)shape->cache_head_stride * 2 : (cuuint64_t)D * 2;
+    const cuuint64_t ls = shape->num_layers > 1 ? (cuuint64_t)shape->cache_layer_stride * 2
+                                                : (cuuint64_t)shape->cache_token_stride * 2 * shape->total_tokens;
+    const cuuint64_t strides[3] = {hs, (cuuint64_t)shape->cache_token_stride * 2, ls};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)kTileKeys, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = encode(&tmap_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k_cache), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cuda_fail((int)r);
+  }
+
+  ScoreParams p;
+  p.cu = shape->cu_seqlens;
+  p.importance = importance;
+  p.part_m = static_cast<float*>(workspace);
+  p.part_l = p.part_m + (size_t)shape->num_layers * shape->num_kv_heads * pl.max_items * pl.Ralloc;
+  p.dev_status = dev_status;
+  p.T = shape->total_tokens;
+  p.B = shape->batch;
+  p.Hkv = shape->num_kv_heads;
+  p.G = G;
+  p.W = shape->window;
+  p.R = pl.R;
+  p.Rpad = pl.Rpad;
+  p.Ralloc = pl.Ralloc;
+  p.tiles_per_chunk = pl.tiles_per_chunk;
+  p.max_items = pl.max_items;
+  p.k_stages = pl.k_stages;
+  p.scale_log2 = kLog2e / sqrtf((float)D);
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const dim3 grid((unsigned)pl.max_items, (unsigned)shape->num_kv_heads, (unsigned)shape->num_layers);
+#define SG_LAUNCH_SCORE(DD, P1)                                                                                      \
+  do {                                                                                                               \
+    SG_CUDA_TRY(cudaFuncSetAttribute(score_kernel<DD, P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes)); \
+    score_kernel<DD, P1><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);                               \
+    SG_CUDA_TRY(cudaGetLastError());                                                                                 \
+  } while (0)
+  if (D == 128) { SG_LAUNCH_SCORE(128, true); SG_LAUNCH_SCORE(128, false); }
+  else          { SG_LAUNCH_SCORE(64, true);  SG_LAUNCH_SCORE(64, false); }
+#undef SG_LAUNCH_SCORE
+  return SG_OK;
 }
