@@ -1,0 +1,446 @@
+#!/usr/bin/env python
+"""Benchmark of the selective-KV hot path on B200: score -> select -> pack -> sparse decode.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2|c4|c3|c5]
+
+One "step" is one pass of the whole path over one batch of synthetic prompts: sg_score,
+sg_select_topk and sg_pack_kv over all layers (one call each), then the workload's decode steps
+(one sg_sparse_decode_attn call per layer per step, replayed from a CUDA graph).  The default
+workload is the Llama-3-8B-shaped cache (32 layers, 8192-token prompt, 10 % budget, 64 decode
+steps).  Rank 0 prints ONE JSON line; see the design doc for the meaning of every key.
+
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "prefill select+pack GB/s (sparse-decode tokens/s in decode_tokens_per_s)"
+UNIT = "GB/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (bytes; None where no capture exists).  Keyed by workload then kernel.
+NCU_TRAFFIC = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_config(name: str, args):
+    from paper_2607_28150_b200 import workloads as wl
+    if name == "c2":
+        return wl.llama8b() if args.layers is None else wl.llama8b(num_layers=args.layers)
+    if name == "c4":
+        return wl.llama70b() if args.layers is None else wl.llama70b(num_layers=args.layers)
+    if name == "c3":
+        return wl.varlen(args.fraction)
+    if name == "c5":
+        return wl.decode_sweep(args.batch, args.sel, args.rho)
+    if name == "c1":
+        return wl.tiny()
+    raise SystemExit("unknown workload %s" % name)
+
+
+def algorithmic_work(cfg, n_loc):
+    """Algorithmic bytes / flops of one step, per stage (what the method must move or compute, counted once)."""
+    L, Hkv, d, G, W = cfg.num_layers, cfg.num_kv_heads, cfg.head_dim, cfg.group, cfg.window
+    lens = np.asarray(cfg.seqlens, dtype=np.int64)
+    ks = cfg.budgets().astype(np.int64)
+    T, Ktot, NL = int(lens.sum()), int(ks.sum()), int(np.sum(n_loc))
+    R = G * W
+    work = {
+        "score": {"flops": float(2 * R * d * T * Hkv * L),
+                  "bytes": float(L * Hkv * (T * d * 2 + T * 4) + L * cfg.batch * W * cfg.num_q_heads * d * 2)},
+        "select": {"bytes": float(L * Hkv * (T * 4 + Ktot * 4))},
+        "pack": {"bytes": float(L * Hkv * Ktot * (2 * 2 * d * 2 + 4))},
+        "decode_call": {"bytes": float(Hkv * (2 * (Ktot + NL) * d * 2 + NL * 4) + 2 * cfg.batch * cfg.num_q_heads * d * 2),
+                        "flops": float(4 * G * d * (Ktot + NL) * Hkv)},
+    }
+    return work
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.strip().split(", ") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, r[4:8]):
+                if val.strip().lower().startswith("active"):
+                    reasons.add(nm)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# --------------------------------------------------------------------------------------------- oracle arm
+def oracle_sample(cfg, layers, n_decode_layers=None):
+    """Time the CPU oracle, as it stands, on `layers` of the workload: score, select, pack, one decode step."""
+    import oracle
+    from paper_2607_28150_b200 import workloads as wl
+    data = wl.make_prefill(cfg, layers)
+    cu, ck = data["cu_seqlens"], cfg.cu_k()
+    t = {}
+    t0 = time.perf_counter(); imp = oracle.score(data["q_win"], data["k"], cu); t["score"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); sel = oracle.select_topk(imp, cu, ck); t["select"] = time.perf_counter() - t0
+    t0 = time.perf_counter(); pk, pv = oracle.pack_kv(data["k"], data["v"], cu, sel, ck); t["pack"] = time.perf_counter() - t0
+    nloc = cfg.n_local()
+    td = 0.0
+    for i, l in enumerate(layers):
+        q = wl.make_decode_queries(cfg, l, 0, data["q_win"][i])
+        _, _, loc, cl = wl.make_index_split(cfg, l, 0, cfg.budgets(), nloc, exclude=sel[i], cu_excl=ck)
+        t0 = time.perf_counter()
+        oracle.sparse_decode_attn(q, pk[i], pv[i], ck, data["k"][i], data["v"][i], cu, loc, cl)
+        td += time.perf_counter() - t0
+    t["decode"] = td
+    return t
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    cfg = workload_config(args.workload, args)
+    layers = list(range(min(2, cfg.num_layers)))
+    work = algorithmic_work(cfg, cfg.n_local())
+    frac = len(layers) / cfg.num_layers
+    for _ in range(args.warmup):
+        oracle_sample(cfg, layers)
+    t_all, t_sp, t_dec = 0.0, 0.0, 0.0
+    for _ in range(args.steps):
+        t0 = time.perf_counter()
+        t = oracle_sample(cfg, layers)
+        t_all += time.perf_counter() - t0
+        t_sp += t["select"] + t["pack"]
+        t_dec += t["decode"]
+    value = (work["select"]["bytes"] + work["pack"]["bytes"]) * frac * args.steps / t_sp / 1e9
+    dec_tok = cfg.batch * len(layers) / cfg.num_layers * args.steps / t_dec
+    cores = oracle.max_threads()
+    sample = "layers 0-%d of %s per step: oracle score+select+pack and one decode step over those layers" % (
+        layers[-1], cfg.name)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "sample": sample},
+            "decode_tokens_per_s": dec_tok,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_28150_b200 import binding as sg, workloads as wl
+    from paper_2607_28150_b200.pipeline import HotPath
+
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+    cfg = workload_config(args.workload, args)
+    L, B, Hq, Hkv, d, W = cfg.num_layers, cfg.batch, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.window
+    T = cfg.total_tokens
+    nsteps_dec = args.decode_steps if args.decode_steps is not None else cfg.decode_steps
+    nloc = cfg.n_local()
+    cu_nloc_h = np.concatenate([[0], np.cumsum(nloc)]).astype(np.int32)
+    NL = int(cu_nloc_h[-1])
+    work = algorithmic_work(cfg, nloc)
+
+    # ---- synthetic inputs: generated on the host (seeded), kept in pinned memory for the end-to-end arm
+    t_gen = time.perf_counter()
+    h_q = torch.empty((L, B, W, Hq, d), dtype=torch.int16).pin_memory()
+    h_k = torch.empty((L, T, Hkv, d), dtype=torch.int16).pin_memory()
+    h_v = torch.empty((L, T, Hkv, d), dtype=torch.int16).pin_memory()
+    for l in range(L):
+        lay = wl.make_layer(cfg, l)
+        h_q[l] = torch.from_numpy(lay["q_win"].view(np.int16))
+        h_k[l] = torch.from_numpy(lay["k"].view(np.int16))
+        h_v[l] = torch.from_numpy(lay["v"].view(np.int16))
+    d_q, d_k, d_v = h_q.to(dev), h_k.to(dev), h_v.to(dev)
+    hp = HotPath(L, Hq, Hkv, d, W, cfg.seqlens, cfg.budgets(), device=dev)
+    Ktot = hp.K_tot
+
+    # one untimed pass to obtain the selected sets, from which the local (on-demand) indices are drawn
+    hp.prefill(d_q, d_k, d_v)
+    torch.cuda.synchronize()
+    sel_host = hp.sel_idx.cpu().numpy()
+    h_qdec = torch.empty((nsteps_dec, L, B, Hq, d), dtype=torch.int16).pin_memory()
+    h_idx = torch.empty((nsteps_dec, L, Hkv, max(NL, 1)), dtype=torch.int32).pin_memory()
+    qwin_f = [wl.bf16_bits_to_f32(h_q[l].numpy().view(np.uint16)).mean(axis=1) for l in range(L)]
+    for s in range(nsteps_dec):
+        rng = np.random.Generator(np.random.Philox(key=1000 * cfg.config_id + 7 + 100000 * (s + 1)))
+        qd = rng.standard_normal((L, B, Hq, d), dtype=np.float32) + np.stack(qwin_f)
+        h_qdec[s] = torch.from_numpy(wl.f32_to_bf16_bits(qd).view(np.int16))
+    if NL:
+        ck = hp.cu_k_host
+        for l in range(L):
+            rng = np.random.Generator(np.random.Philox(key=1000 * cfg.config_id + 10 * l + 6))
+            for b, n in enumerate(cfg.seqlens):
+                if nloc[b] == 0:
+                    continue
+                for g in range(Hkv):
+                    rest = np.setdiff1d(np.arange(n, dtype=np.int32), sel_host[l, g, ck[b]:ck[b + 1]])
+                    draws = rng.permuted(np.tile(rest, (nsteps_dec, 1)), axis=1)[:, : nloc[b]]
+                    h_idx[:, l, g, cu_nloc_h[b]:cu_nloc_h[b + 1]] = torch.from_numpy(draws)
+    d_qdec, d_idx = h_qdec.to(dev), h_idx.to(dev)
+    d_cu_nloc = torch.from_numpy(cu_nloc_h).to(dev)
+    d_out = torch.empty((nsteps_dec, L, B, Hq, d), dtype=torch.bfloat16, device=dev)
+    h_out = torch.empty((nsteps_dec, L, B, Hq, d), dtype=torch.bfloat16).pin_memory()
+    h_pk = torch.empty(hp.packed_k.shape, dtype=torch.int16).pin_memory()
+    h_pv = torch.empty(hp.packed_v.shape, dtype=torch.int16).pin_memory()
+    h_sel = torch.empty(hp.sel_idx.shape, dtype=torch.int32).pin_memory()
+    hp.decode_workspace(NL)
+    gen_s = time.perf_counter() - t_gen
+
+    def decode_all(with_copies: bool):
+        for s in range(nsteps_dec):
+            if with_copies:
+                d_qdec[s].copy_(h_qdec[s], non_blocking=True)
+                if NL:
+                    d_idx[s].copy_(h_idx[s], non_blocking=True)
+            for l in range(L):
+                hp.decode(l, d_qdec[s, l], d_k[l], d_v[l], d_idx[s, l] if NL else None, d_cu_nloc, NL, d_out[s, l])
+            if with_copies:
+                h_out[s].copy_(d_out[s], non_blocking=True)
+
+    # eager once (sets kernel attributes), then capture both decode graphs
+    if nsteps_dec:
+        hp.decode(0, d_qdec[0, 0], d_k[0], d_v[0], d_idx[0, 0] if NL else None, d_cu_nloc, NL, d_out[0, 0])
+    torch.cuda.synchronize()
+    g_res, g_e2e = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    if nsteps_dec:
+        with torch.cuda.graph(g_res):
+            decode_all(False)
+        with torch.cuda.graph(g_e2e):
+            decode_all(True)
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+
+    def step(e2e: bool, ev):
+        """One pass of the path.  `ev` is a list of 6 events bracketing: h2d | score | select | pack | d2h | decode."""
+        ev[0].record(stream)
+        if e2e:
+            d_q.copy_(h_q, non_blocking=True); d_k.copy_(h_k, non_blocking=True); d_v.copy_(h_v, non_blocking=True)
+        ev[1].record(stream)
+        hp.score(d_q, d_k)
+        ev[2].record(stream)
+        hp.select()
+        ev[3].record(stream)
+        hp.pack(d_k, d_v)
+        ev[4].record(stream)
+        if e2e:
+            h_pk.copy_(hp.packed_k, non_blocking=True); h_pv.copy_(hp.packed_v, non_blocking=True)
+            h_sel.copy_(hp.sel_idx, non_blocking=True)
+        ev[5].record(stream)
+        if nsteps_dec:
+            (g_e2e if e2e else g_res).replay()
+        ev[6].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(e2e: bool, steps: int, warmup: int):
+        mk = lambda: [torch.cuda.Event(enable_timing=True) for _ in range(7)]
+        for _ in range(warmup):
+            step(e2e, mk())
+        evs = [mk() for _ in range(steps)]
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for i in range(steps):
+            step(e2e, evs[i])
+        t1.record(stream)
+        barrier()
+        total_ms = t0.elapsed_time(t1)
+        names = ["h2d", "score", "select", "pack", "d2h", "decode"]
+        stage = {n: sum(e[i].elapsed_time(e[i + 1]) for e in evs) / steps for i, n in enumerate(names)}
+        if world > 1:
+            tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            total_ms = float(tt.item())
+        return total_ms / steps, stage
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_step, st = timed(False, args.steps, max(3, args.warmup))
+    clocks = sampler.stop() if rank == 0 else {}
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    ms_e2e, st_e = timed(True, e2e_steps, 1)
+    status = hp.read_status()
+
+    if world > 1:
+        gather = [None] * world
+        dist.all_gather_object(gather, {"st": st, "st_e": st_e})
+        st = {k: max(gg["st"][k] for gg in gather) for k in st}
+        st_e = {k: max(gg["st_e"][k] for gg in gather) for k in st_e}
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    sp_bytes = work["select"]["bytes"] + work["pack"]["bytes"]
+    value = world * sp_bytes / ((st["select"] + st["pack"]) * 1e-3) / 1e9
+    dec_tok = world * B * nsteps_dec / (st["decode"] * 1e-3) if nsteps_dec else None
+    e2e_value = world * sp_bytes / ((st_e["h2d"] + st_e["select"] + st_e["pack"] + st_e["d2h"]) * 1e-3) / 1e9
+    e2e_dec_tok = world * B * nsteps_dec / (st_e["decode"] * 1e-3) if nsteps_dec else None
+    h2d = (h_q.numel() + h_k.numel() + h_v.numel()) * 2 + (h_qdec.numel() * 2 + (h_idx.numel() * 4 if NL else 0))
+    d2h = (h_pk.numel() + h_pv.numel()) * 2 + h_sel.numel() * 4 + h_out.numel() * 2
+
+    # ---- rooflines, per kernel class, from the stage times of the device-resident arm
+    ncalls_dec = nsteps_dec * L
+    tc_peak = peaks["bf16_tflops_sustained"]
+    ncu = NCU_TRAFFIC.get(args.workload, {})
+    def hbm(name, nbytes, ms, launches):
+        a = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+        return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy)", "ms_per_step": ms,
+                "launches_per_step": launches, "traffic": ncu.get(name)}
+    roofs = {
+        "score": hbm("score", work["score"]["bytes"], st["score"], 2),
+        "select": hbm("select", work["select"]["bytes"], st["select"], 1),
+        "pack": hbm("pack", work["pack"]["bytes"], st["pack"], 1),
+    }
+    roofs["score"]["tensor_tflops"] = work["score"]["flops"] / (st["score"] * 1e-3) / 1e12
+    roofs["score"]["tensor_frac_of_sustained"] = roofs["score"]["tensor_tflops"] / tc_peak
+    R = cfg.group * W
+    if R > peaks["bf16_tflops_sustained"] * 1e3 / peaks["hbm_gbs"]:       # above the ridge: tensor cores bind
+        roofs["score"].update(bound="tensor", achieved=roofs["score"]["tensor_tflops"], peak=tc_peak, unit="TFLOP/s",
+                              frac=roofs["score"]["tensor_frac_of_sustained"], peak_source=peaks["source"] + " (sustained bf16)")
+    if ncalls_dec:
+        roofs["decode"] = hbm("decode", work["decode_call"]["bytes"] * ncalls_dec, st["decode"], 2 * ncalls_dec)
+        roofs["decode"]["us_per_call"] = 1e3 * st["decode"] / ncalls_dec
+    dominant = max(roofs.values(), key=lambda r: r["ms_per_step"])
+
+    # ---- the oracle on the host cores, bounded sample
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        layers = list(range(min(4, L)))
+        t = oracle_sample(cfg, layers)
+        fr = len(layers) / L
+        cpu = {"value": sp_bytes * fr / (t["select"] + t["pack"]) / 1e9, "unit": UNIT, "cores": oracle.max_threads(),
+               "kind": "oracle",
+               "sample": "layers 0-%d of %s: score %.2fs, select %.3fs, pack %.3fs, one decode step %.3fs" % (
+                   layers[-1], cfg.name, t["score"], t["select"], t["pack"], t["decode"]),
+               "decode_tokens_per_s": B * fr / t["decode"] if t["decode"] > 0 else None,
+               "score_tflops": work["score"]["flops"] * fr / t["score"] / 1e12}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "%s: L=%d B=%d Hq=%d Hkv=%d d=%d W=%d T=%d K_tot=%d n_loc=%d decode_steps=%d" % (
+                       cfg.name, L, B, Hq, Hkv, d, W, T, Ktot, NL, nsteps_dec),
+                   "l2": "inputs larger than L2 (K+V caches %.0f MiB); no flush" % ((h_k.numel() + h_v.numel()) * 2 / 2**20),
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "decode": "one sg_sparse_decode_attn call per layer per step, replayed from a CUDA graph"},
+        "decode_tokens_per_s": dec_tok,
+        "stage_ms": st,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
+        "gpu_launches": args.steps * (4 + 2 * ncalls_dec),
+        "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
+        "dev_status": status, "setup_s": gen_s,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--fraction", type=float, default=0.10, help="c3: budget fraction")
+    ap.add_argument("--batch", type=int, default=64, help="c5: concurrent sequences")
+    ap.add_argument("--sel", type=float, default=0.2, help="c5: required fraction of the prompt")
+    ap.add_argument("--rho", type=float, default=0.25, help="c5: index-addressed share of the required entries")
+    ap.add_argument("--layers", type=int, default=None, help="c2/c4: override the number of layers (small profiling cases)")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

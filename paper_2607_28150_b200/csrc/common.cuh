@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "smartgen.h"
 
 namespace sg {
@@ -24,6 +26,19 @@ inline sg_status cuda_fail(int err) {
   do {                                                           \
     cudaError_t _e = (expr);                                     \
     if (_e != cudaSuccess) return ::sg::cuda_fail((int)_e);      \
+  } while (0)
+
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device and call site (the setting is
+// sticky per device, so later calls -- including calls made during stream capture -- skip the driver).
+#define SG_ENSURE_SMEM(func, bytes)                                                                   \
+  do {                                                                                                \
+    static std::atomic<int> _sg_set[64];                                                              \
+    int _sg_dev = 0;                                                                                  \
+    SG_CUDA_TRY(cudaGetDevice(&_sg_dev));                                                             \
+    if (_sg_dev < 0 || _sg_dev >= 64 || _sg_set[_sg_dev].load(std::memory_order_relaxed) < (bytes)) { \
+      SG_CUDA_TRY(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (bytes)));  \
+      if (_sg_dev >= 0 && _sg_dev < 64) _sg_set[_sg_dev].store((bytes), std::memory_order_relaxed);   \
+    }                                                                                                 \
   } while (0)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

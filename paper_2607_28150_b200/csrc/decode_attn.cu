@@ -467,8 +467,7 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   const dim3 grid2((unsigned)shape->num_q_heads, (unsigned)shape->batch);
 #define SG_LAUNCH_DECODE(DD, HI)                                                                                \
   do {                                                                                                          \
-    SG_CUDA_TRY(cudaFuncSetAttribute(decode_partial_kernel<DD, HI>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                     decode_smem_bytes<DD>()));                                                 \
+    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI>), decode_smem_bytes<DD>());                                   \
     decode_partial_kernel<DD, HI><<<grid1, kDecThreads, decode_smem_bytes<DD>(), s>>>(p);                        \
   } while (0)
   if (total_sel + total_loc > 0) {

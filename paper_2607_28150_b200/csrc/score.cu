@@ -594,7 +594,7 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   const dim3 grid((unsigned)pl.max_items, (unsigned)shape->num_kv_heads, (unsigned)shape->num_layers);
 #define SG_LAUNCH_SCORE(DD, P1)                                                                                      \
   do {                                                                                                               \
-    SG_CUDA_TRY(cudaFuncSetAttribute(score_kernel<DD, P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes)); \
+    SG_ENSURE_SMEM((score_kernel<DD, P1>), pl.smem_bytes);                                                           \
     score_kernel<DD, P1><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);                               \
     SG_CUDA_TRY(cudaGetLastError());                                                                                 \
   } while (0)

@@ -191,7 +191,7 @@ extern "C" sg_status sg_select_topk(const sg_shape* shape, const float* importan
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (shape->max_seqlen <= kSelKeyCap) {
     const int smem = kSelFixedSmem + shape->max_seqlen * 4;
-    SG_CUDA_TRY(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    SG_ENSURE_SMEM(select_topk_kernel<true>, smem);
     select_topk_kernel<true><<<(unsigned)rows, kSelThreads, smem, s>>>(p);
   } else {
     select_topk_kernel<false><<<(unsigned)rows, kSelThreads, kSelFixedSmem, s>>>(p);
