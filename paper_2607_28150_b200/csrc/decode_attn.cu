@@ -7,8 +7,14 @@
 // conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).
 // Each warp owns 16 tokens of a tile: S = Q K^T and O += P V run on bf16 tensor-core MMAs with the
 // G query rows of the KV head padded to 16, the online softmax (base 2) stays in registers.
-// Per-chunk partials (m, l, unnormalised O) go to the workspace; a second kernel merges them with
-// the log-sum-exp rule and writes bf16 out and fp32 lse.
+// The split-KV partials (m, l, unnormalised O) are merged with the log-sum-exp rule in one of two ways:
+//   fused  -- the CTAs that share a (sequence, KV head) form a thread-block cluster; each leaves its
+//             partial in its own shared memory and, after a cluster barrier, every CTA merges a slice
+//             of the output through distributed shared memory.  One launch, no workspace traffic.
+//   two-kernel -- partials go to the workspace and a second kernel merges them; used when a few very
+//             long token lists need more CTAs than a cluster can hold.
+// Both launches use programmatic dependent launch, so back-to-back decode calls overlap their
+// launch latency and prologue with the previous call's tail.
 #include "common.cuh"
 #include "launch.h"
 
@@ -40,6 +46,7 @@ struct DecParams {
   int32_t* dev_status;
   int64_t ts, hs;
   int32_t B, Hq, Hkv, G, K_tot, NL_tot, chunk;
+  int32_t csize;     // fused mode: CTAs per (sequence, KV head) = cluster size
   float scale_log2;
 };
 
@@ -99,8 +106,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ float ld_dsmem_f32(const float* local_ptr, uint32_t cta_rank) {
+  uint32_t remote;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
+// Programmatic dependent launch: let the next kernel in the stream start its prologue now, and wait
+// for the previous kernel's memory before touching anything it may have written.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // kHi: the KV head has more than 8 query rows, so MMA rows 8..15 carry data too.
-template <int D, bool kHi>
+// kFused: the CTAs of a (sequence, KV head) form a cluster and merge their partials through DSMEM.
+template <int D, bool kHi, bool kFused>
 __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const DecParams p) {
   constexpr int kRowBytes = D * 2;
   constexpr int kChunksPerRow = D / 8;                       // 16-byte chunks
@@ -113,28 +136,23 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
+  pdl_launch_dependents();
+  pdl_wait();
   int b, c;
-  if (!find_item(p, blockIdx.x, lane, b, c)) return;
+  if (kFused) {
+    b = blockIdx.z;
+    c = blockIdx.x;                                            // rank in the cluster
+  } else if (!find_item(p, blockIdx.x, lane, b, c)) {
+    return;
+  }
   const int kb = p.cu_k[b + 1] - p.cu_k[b];
   const int nl = p.cu_nloc[b + 1] - p.cu_nloc[b];
   const int c0 = p.cu[b];
   const int nseq = p.cu[b + 1] - c0;
-  const int pos_beg = c * p.chunk;
-  const int pos_end = min(kb + nl, pos_beg + p.chunk);
-  const int ntok = pos_end - pos_beg;
-  const int ntiles = (ntok + kTile - 1) / kTile;
-
-  // Stage this chunk's local indices (validated); packed positions get 0.
-  for (int i = tid; i < ntok; i += kDecThreads) {
-    const int pos = pos_beg + i;
-    int v = 0;
-    if (pos >= kb) {
-      v = __ldg(p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + (pos - kb));
-      if (v < 0 || v >= nseq) { v = -1; raise(p.dev_status, SG_ERR_INDEX); }
-    }
-    s_idx[i] = v;
-  }
-  __syncthreads();
+  // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
+  const int span = kFused ? ((((kb + nl + p.csize - 1) / p.csize) + kTile - 1) / kTile) * kTile : p.chunk;
+  const int range_beg = min(kb + nl, c * span);
+  const int range_end = min(kb + nl, range_beg + span);
 
   const uint16_t* pk_base = p.packed_k + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
   const uint16_t* pv_base = p.packed_v + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
@@ -142,6 +160,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   const uint16_t* lv_base = p.local_v + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
   const uint32_t sk_u32 = smem_u32(sk), sv_u32 = smem_u32(sv);
 
+  int pos_beg = 0, ntok = 0;                                   // current sub-chunk (at most kMaxChunk tokens)
   auto load_tile = [&](int tile, int stage) {
 #pragma unroll
     for (int i = 0; i < kCopiesPerThread; ++i) {
@@ -193,6 +212,21 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   for (int i = 0; i < D / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
+#pragma unroll 1
+  for (pos_beg = range_beg; pos_beg < range_end; pos_beg += kMaxChunk) {
+  ntok = min(range_end - pos_beg, kMaxChunk);
+  const int ntiles = (ntok + kTile - 1) / kTile;
+  // Stage this sub-chunk's local indices (validated); packed positions get 0.
+  for (int i = tid; i < ntok; i += kDecThreads) {
+    const int pos = pos_beg + i;
+    int v = 0;
+    if (pos >= kb) {
+      v = __ldg(p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + (pos - kb));
+      if (v < 0 || v >= nseq) { v = -1; raise(p.dev_status, SG_ERR_INDEX); }
+    }
+    s_idx[i] = v;
+  }
+  __syncthreads();
 #pragma unroll
   for (int s = 0; s < kStages - 1; ++s) {
     if (s < ntiles) load_tile(s, s);
@@ -306,6 +340,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   }
   cp_async_wait<0>();
   __syncthreads();
+  }  // sub-chunks
 
   // merge the four warps through shared memory (the pipeline buffers are free now)
   float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
@@ -323,6 +358,9 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     if (kHi) { dst[8 * D] = o_acc[i][2]; dst[8 * D + 1] = o_acc[i][3]; }
   }
   __syncthreads();
+  float* sm_co = sm_l + kDecWarps * 16;                       // CTA-level partial: O [16][D], m [16], l [16]
+  float* sm_cm = sm_co + 16 * D;
+  float* sm_cl = sm_cm + 16;
   const int64_t slot = (int64_t)blockIdx.x * p.Hkv + g;
   float* po = p.part_o + slot * p.G * D;
   float* pml = p.part_ml + slot * p.G * 2;
@@ -339,8 +377,37 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
       L += sm_l[w * 16 + r] * f;
       O += sm_o[(w * 16 + r) * D + col] * f;
     }
-    po[e] = O;
-    if (col == 0) { pml[2 * r] = M; pml[2 * r + 1] = L; }
+    if (kFused) {
+      sm_co[e] = O;
+      if (col == 0) { sm_cm[r] = M; sm_cl[r] = L; }
+    } else {
+      po[e] = O;
+      if (col == 0) { pml[2 * r] = M; pml[2 * r + 1] = L; }
+    }
+  }
+  if (kFused) {
+    // Every CTA of the cluster merges a slice of the G*D outputs, reading all ranks' partials.
+    const int cs = p.csize;
+    if (cs > 1) cluster_sync_all(); else __syncthreads();
+    const int per = (p.G * D + cs - 1) / cs;
+    const int e_beg = c * per, e_end = min(p.G * D, e_beg + per);
+    __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
+    for (int e = e_beg + tid; e < e_end; e += kDecThreads) {
+      const int r = e / D, col = e - r * D;
+      float M = -INFINITY;
+      for (int j = 0; j < cs; ++j) M = fmaxf(M, cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r]);
+      const float Mu = M == -INFINITY ? 0.f : M;
+      float L = 0.f, O = 0.f;
+      for (int j = 0; j < cs; ++j) {
+        const float mj = cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r];
+        const float f = exp2f(mj - Mu);
+        L += (cs > 1 ? ld_dsmem_f32(sm_cl + r, j) : sm_cl[r]) * f;
+        O += (cs > 1 ? ld_dsmem_f32(sm_co + e, j) : sm_co[e]) * f;
+      }
+      outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+      if (p.lse && col == 0) p.lse[(int64_t)b * p.Hq + (int64_t)g * p.G + r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    }
+    if (cs > 1) cluster_sync_all();                           // keep every CTA's shared memory alive until all reads are done
   }
 }
 
@@ -350,6 +417,8 @@ template <int D>
 __global__ void __launch_bounds__(D) decode_combine_kernel(const DecParams p) {
   __shared__ int s_part[D / 32];
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int g = h / p.G, r = h - g * p.G;
   // first work item of sequence b = number of chunks of the sequences before it
   int cnt = 0;
@@ -397,13 +466,29 @@ int decode_chunk_tokens(const sg_shape* shape, int32_t total_sel, int32_t total_
   return (int)chunk;
 }
 
+// Fused (cluster) mode: CTAs per (sequence, KV head), a power of two <= 8; 0 selects the two-kernel mode.
+// The fused mode is used unless there are too few (sequence, head) pairs to fill the GPU with clusters of
+// 8 while each list is long enough to feed many more CTAs.
+int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
+  const int64_t pairs = (int64_t)shape->batch * shape->num_kv_heads;
+  if (shape->batch > 65535) return 0;
+  const int64_t avg_tiles = (((int64_t)total_sel + total_loc) / shape->batch + kTile - 1) / kTile;
+  if (pairs * 8 < kNumSMs && avg_tiles >= 64) return 0;
+  int by_work = 1;
+  while (by_work < 8 && by_work * 2 * 2 <= avg_tiles) by_work *= 2;        // at least two tiles per CTA
+  int by_fill = 1;
+  while (by_fill < 8 && pairs * by_fill < 2 * kNumSMs) by_fill *= 2;        // about two CTAs per SM
+  return by_work < by_fill ? by_work : by_fill;
+}
+
 static int64_t decode_max_items(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
   const int chunk = decode_chunk_tokens(shape, total_sel, total_loc);
   return ((int64_t)total_sel + total_loc + chunk - 1) / chunk + shape->batch;
 }
 
 size_t decode_workspace_bytes(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
-  if (shape->num_kv_heads < 1 || shape->num_q_heads < 1) return 0;
+  if (shape->num_kv_heads < 1 || shape->num_q_heads < 1 || shape->batch < 1) return 0;
+  if (decode_cluster_size(shape, total_sel, total_loc) > 0) return 0;       // fused mode keeps partials on chip
   const int64_t items = decode_max_items(shape, total_sel, total_loc);
   const int G = shape->num_q_heads / shape->num_kv_heads;
   return (size_t)items * shape->num_kv_heads * G * (shape->head_dim + 2) * sizeof(float);
@@ -429,9 +514,6 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
       !aligned16(workspace) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
     return SG_ERR_INVALID;
   if (!(softmax_scale >= 0.f)) return SG_ERR_INVALID;
-  const size_t need = decode_workspace_bytes(shape, total_sel, total_loc);
-  if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
-
   const int D = shape->head_dim;
   const int G = shape->num_q_heads / shape->num_kv_heads;
   const int64_t items = decode_max_items(shape, total_sel, total_loc);
@@ -446,8 +528,8 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.cu_k = cu_k;
   p.cu_nloc = cu_nloc;
   p.local_idx = local_idx;
-  p.part_o = static_cast<float*>(workspace);
-  p.part_ml = p.part_o + items * shape->num_kv_heads * G * D;
+  p.part_o = nullptr;
+  p.part_ml = nullptr;
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.dev_status = dev_status;
@@ -463,21 +545,52 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const dim3 grid1((unsigned)items, (unsigned)shape->num_kv_heads);
-  const dim3 grid2((unsigned)shape->num_q_heads, (unsigned)shape->batch);
-#define SG_LAUNCH_DECODE(DD, HI)                                                                                \
-  do {                                                                                                          \
-    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI>), decode_smem_bytes<DD>());                                   \
-    decode_partial_kernel<DD, HI><<<grid1, kDecThreads, decode_smem_bytes<DD>(), s>>>(p);                        \
+  p.csize = decode_cluster_size(shape, total_sel, total_loc);
+  const bool fused = p.csize > 0;
+
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[0].val.programmaticStreamSerializationAllowed = 1;
+  attrs[1].id = cudaLaunchAttributeClusterDimension;
+  attrs[1].val.clusterDim.x = fused ? (unsigned)p.csize : 1u;
+  attrs[1].val.clusterDim.y = 1;
+  attrs[1].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = s;
+  cfg.attrs = attrs;
+  cfg.blockDim = dim3(kDecThreads);
+#define SG_LAUNCH_DECODE(DD, HI, FU)                                                                  \
+  do {                                                                                                \
+    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI, FU>), decode_smem_bytes<DD>());                     \
+    cfg.dynamicSmemBytes = decode_smem_bytes<DD>();                                                   \
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<DD, HI, FU>, p));                      \
   } while (0)
-  if (total_sel + total_loc > 0) {
-    if (D == 128) { if (G > 8) SG_LAUNCH_DECODE(128, true); else SG_LAUNCH_DECODE(128, false); }
-    else          { if (G > 8) SG_LAUNCH_DECODE(64, true);  else SG_LAUNCH_DECODE(64, false); }
-    SG_CUDA_TRY(cudaGetLastError());
+#define SG_LAUNCH_DECODE_D(DD)                                                                        \
+  do {                                                                                                \
+    if (fused) { if (G > 8) SG_LAUNCH_DECODE(DD, true, true); else SG_LAUNCH_DECODE(DD, false, true); } \
+    else       { if (G > 8) SG_LAUNCH_DECODE(DD, true, false); else SG_LAUNCH_DECODE(DD, false, false); } \
+  } while (0)
+  if (fused) {
+    // one launch: grid (cluster size, H_kv, B); sequences with empty lists still get out = 0, lse = -inf
+    cfg.gridDim = dim3((unsigned)p.csize, (unsigned)shape->num_kv_heads, (unsigned)shape->batch);
+    cfg.numAttrs = p.csize > 1 ? 2 : 1;
+    if (D == 128) SG_LAUNCH_DECODE_D(128); else SG_LAUNCH_DECODE_D(64);
+    return SG_OK;
   }
+  const size_t need = decode_workspace_bytes(shape, total_sel, total_loc);
+  if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
+  p.part_o = static_cast<float*>(workspace);
+  p.part_ml = p.part_o + items * shape->num_kv_heads * G * D;
+  cfg.numAttrs = 1;
+  if (total_sel + total_loc > 0) {
+    cfg.gridDim = dim3((unsigned)items, (unsigned)shape->num_kv_heads);
+    if (D == 128) SG_LAUNCH_DECODE_D(128); else SG_LAUNCH_DECODE_D(64);
+  }
+#undef SG_LAUNCH_DECODE_D
 #undef SG_LAUNCH_DECODE
-  if (D == 128) decode_combine_kernel<128><<<grid2, 128, 0, s>>>(p);
-  else decode_combine_kernel<64><<<grid2, 64, 0, s>>>(p);
-  SG_CUDA_TRY(cudaGetLastError());
+  cfg.gridDim = dim3((unsigned)shape->num_q_heads, (unsigned)shape->batch);
+  cfg.dynamicSmemBytes = 0;
+  if (D == 128) { cfg.blockDim = dim3(128); SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<128>, p)); }
+  else          { cfg.blockDim = dim3(64);  SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<64>, p)); }
   return SG_OK;
 }

@@ -43,11 +43,14 @@ def test_host_side_argument_checks_need_no_gpu():
     bad = ctypes.c_void_p(0x1004)        # misaligned
     assert lib.sg_pack_kv(ctypes.byref(s), bad, fake, fake, fake, 4, fake, fake, None, None) == sg.SG_ERR_INVALID
     assert lib.sg_pack_kv(ctypes.byref(s), fake, fake, fake, fake, -1, fake, fake, None, None) == sg.SG_ERR_INVALID
-    # decode: workspace too small is reported before any launch
+    # decode, long lists on few heads (the two-kernel mode): workspace too small is reported before any launch
     lib.sg_sparse_decode_attn.restype = ctypes.c_int
     lib.sg_sparse_decode_attn.argtypes = sg._lib.sg_sparse_decode_attn.argtypes
-    rc = lib.sg_sparse_decode_attn(ctypes.byref(s), fake, fake, fake, fake, 4, fake, fake, fake, fake, 4, 0.0, fake,
-                                   None, fake, 16, None, None)
+    s = sg.Shape(1, 1, 8, 2, 128, 4, 16384, 16384, 0x1000, 16384 * 256, 256, 128)
+    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 8192, 4096) > 16
+    rc = lib.sg_sparse_decode_attn(ctypes.byref(s), fake, fake, fake, fake, 8192, fake, fake, fake, fake, 4096, 0.0,
+                                   fake, None, fake, 16, None, None)
     assert rc == sg.SG_ERR_WORKSPACE
-    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 4, 4) > 16
+    # short lists are merged on chip (cluster mode) and need no workspace
+    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 64, 64) == 0
     assert sg.sg_workspace_bytes(sg.SG_OP_PACK_KV, s, 4, 4) == 0

@@ -47,6 +47,9 @@ def compare(args, **kw):
     ((4096,) * 3, (100, 4096, 1), (3996, 0, 0), 8, 8, 128),   # G = 1, full budget, single token
     ((2000,), (333,), (100,), 32, 2, 128),                    # G = 16
     ((513,), (65,), (63,), 16, 2, 64),                        # G = 8, d = 64, ragged tiles
+    ((12000,), (5000,), (3333,), 8, 2, 128),                  # few heads, long lists: two-kernel split-KV mode
+    ((9000, 100), (4100, 10), (4500, 90), 4, 1, 128),         # two-kernel mode, ragged
+    ((25000,) * 3, (12000,) * 3, (8000,) * 3, 8, 8, 128),     # cluster mode, CTA ranges longer than the index staging buffer
 ])
 def test_decode_matches_oracle(lens, ks, nls, Hq, Hkv, d):
     compare(build(0, lens, ks, nls, Hq, Hkv, d))
