@@ -81,7 +81,7 @@ size_t sg_workspace_bytes(int op, const sg_shape* shape, int32_t total_sel, int3
  * q_win       bf16 [L][B][W][H_q][d], dense; row i of sequence b is the query at N_b - W_eff + i.
  * k_cache     bf16, element (l, token, g, c) at l*layer_stride + token*token_stride + g*head_stride + c.
  * importance  fp32 [L][H_kv][T], fully overwritten.
- * Supported: G*W <= 512 and a multiple of 16 (d = 128) or <= 1024 (d = 64).
+ * Supported: G*W <= 512 (d = 128) or <= 1024 (d = 64), W <= 256.
  */
 sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
@@ -148,6 +148,33 @@ sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void
                                 const int32_t* cu_nloc, int32_t total_loc, float softmax_scale,
                                 void* out, float* lse, void* workspace, size_t workspace_bytes,
                                 int32_t* dev_status, void* stream);
+
+/*
+ * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.
+ *
+ * The paper has no counterpart to this call: it computes exactly what sg_score computes.  It exists
+ * for hosts of this library that may not call cudaMalloc (or any allocating routine) at the point
+ * where they score -- code running under a fixed memory plan, inside a region where allocation is
+ * forbidden, or in a process whose allocator belongs to another runtime.  The scratch that pass 1
+ * and pass 2 of the scoring kernel exchange lives in a fixed array inside the library image,
+ * SG_SCORE_STATIC_SCRATCH_BYTES long; every GPU that loads the library holds that much memory until
+ * the process exits.
+ *
+ *   - Shapes whose sg_workspace_bytes(SG_OP_SCORE, ...) exceeds SG_SCORE_STATIC_SCRATCH_BYTES are
+ *     rejected with SG_ERR_WORKSPACE before anything is launched; use sg_score for those.
+ *   - The call allocates nothing and frees nothing.  The first call on each device looks up the
+ *     array's device address (one cudaGetSymbolAddress with that device current); make that first
+ *     call before starting any stream capture on the device.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  Nothing
+ *     in it needs clearing (every slot is written before it is read within a call), but two calls
+ *     that overlap on the GPU -- different streams, or one stream's call still running when another
+ *     starts -- race on it and give undefined importance.  Serialise them, or use sg_score with
+ *     separate workspaces.
+ *   - Inputs, outputs, status word and error behaviour are those of sg_score.
+ */
+#define SG_SCORE_STATIC_SCRATCH_BYTES (8u << 20)
+sg_status sg_score_static(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
+                          int32_t* dev_status, void* stream);
 
 /* Static description of a status code. */
 const char* sg_strerror(sg_status status);

@@ -21,7 +21,8 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_strerror", "sg_last_cuda_error")
+            "sg_score_static", "sg_strerror", "sg_last_cuda_error")
+SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
     raise ImportError("libsmartgen.so is not built (%s): run `python __graft_entry__.py` or "
@@ -56,6 +57,8 @@ _lib.sg_workspace_bytes.restype = _sz
 _lib.sg_workspace_bytes.argtypes = [ctypes.c_int, _sp, _i32, _i32]
 _lib.sg_score.restype = ctypes.c_int
 _lib.sg_score.argtypes = [_sp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.sg_score_static.restype = ctypes.c_int
+_lib.sg_score_static.argtypes = [_sp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_select_topk.restype = ctypes.c_int
 _lib.sg_select_topk.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _sz, _vp, _vp]
 _lib.sg_pack_kv.restype = ctypes.c_int
@@ -141,6 +144,19 @@ def sg_score(shape: Shape, q_win: torch.Tensor, k_cache: torch.Tensor, importanc
                        _ptr(dev_status), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_score")
+
+
+def sg_score_static(shape: Shape, q_win: torch.Tensor, k_cache: torch.Tensor, importance: torch.Tensor,
+                    dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """`sg_score` for callers that cannot allocate device memory: the scratch between the two scoring
+    passes is a fixed array inside the library (SG_SCORE_STATIC_SCRATCH_BYTES), shared by all calls on a
+    device, so calls must not overlap on the GPU.  Shapes that need more scratch raise SG_ERR_WORKSPACE."""
+    _check(q_win, _BF16, "q_win"); _check(k_cache, _BF16, "k_cache"); _check(importance, torch.float32, "importance")
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_score_static(ctypes.byref(shape), _ptr(q_win), k_cache.data_ptr(), _ptr(importance),
+                              _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_score_static")
 
 
 def sg_select_topk(shape: Shape, importance: torch.Tensor, cu_k: torch.Tensor, total_sel: int,

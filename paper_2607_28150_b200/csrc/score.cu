@@ -603,3 +603,35 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
 #undef SG_LAUNCH_SCORE
   return SG_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// sg_score_static: sg_score for callers that cannot allocate device memory.
+//
+// The row statistics that pass 1 hands to pass 2 normally live in a caller-provided workspace.
+// Here they live in a fixed array that is part of the library image, so the caller needs no
+// allocator at all.  The array is shared by every call on a device and keeps the previous call's
+// contents; nothing in it has to start at zero, because pass 1 writes every slot that pass 2 reads.
+namespace sg {
+namespace {
+static __device__ __align__(256) unsigned char g_score_static_scratch[SG_SCORE_STATIC_SCRATCH_BYTES];
+}  // namespace
+}  // namespace sg
+
+extern "C" sg_status sg_score_static(const sg_shape* shape, const void* q_win, const void* k_cache,
+                                     float* importance, int32_t* dev_status, void* stream) {
+  using namespace sg;
+  sg_status st = check_shape(shape, true);
+  if (st != SG_OK) return st;
+  if (score_workspace_bytes(shape) > (size_t)SG_SCORE_STATIC_SCRATCH_BYTES) return SG_ERR_WORKSPACE;
+  // In host code the array's name is only a handle; the device address has to be asked for, once per
+  // device, with that device current.
+  static std::atomic<void*> scratch_of_device[64];
+  int dev = 0;
+  SG_CUDA_TRY(cudaGetDevice(&dev));
+  void* scratch = (dev >= 0 && dev < 64) ? scratch_of_device[dev].load(std::memory_order_acquire) : nullptr;
+  if (!scratch) {
+    SG_CUDA_TRY(cudaGetSymbolAddress(&scratch, g_score_static_scratch));
+    if (dev >= 0 && dev < 64) scratch_of_device[dev].store(scratch, std::memory_order_release);
+  }
+  return sg_score(shape, q_win, k_cache, importance, scratch, (size_t)SG_SCORE_STATIC_SCRATCH_BYTES, dev_status, stream);
+}
