@@ -7,14 +7,16 @@
 // conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).
 // Each warp owns 16 tokens of a tile: S = Q K^T and O += P V run on bf16 tensor-core MMAs with the
 // G query rows of the KV head padded to 16, the online softmax (base 2) stays in registers.
-// The split-KV partials (m, l, unnormalised O) are merged with the log-sum-exp rule in one of two ways:
-//   fused  -- the CTAs that share a (sequence, KV head) form a thread-block cluster; each leaves its
-//             partial in its own shared memory and, after a cluster barrier, every CTA merges a slice
-//             of the output through distributed shared memory.  One launch, no workspace traffic.
-//   two-kernel -- partials go to the workspace and a second kernel merges them; used when a few very
-//             long token lists need more CTAs than a cluster can hold.
-// Both launches use programmatic dependent launch, so back-to-back decode calls overlap their
-// launch latency and prologue with the previous call's tail.
+// The split-KV partials (m, l, unnormalised O) never leave the chip: the CTAs that share a
+// (sequence, KV head) form a thread-block cluster (1, 2, 4 or 8 CTAs, chosen on the host so that about
+// two CTAs per SM exist and every CTA has at least two tiles); each leaves its partial in its own
+// shared memory and, after a cluster barrier, every CTA merges a slice of the G*d outputs through
+// distributed shared memory with the log-sum-exp rule (m = max m_j, l = sum l_j 2^(m_j-m),
+// o = sum o_j 2^(m_j-m) / l) and writes bf16 out and fp32 lse.  One launch, no workspace.
+// (A two-kernel variant with partials in HBM measured 2x slower on long single-sequence lists and
+// clusters of 16 measured slower than 8 -- few can be co-scheduled -- so neither is kept.)
+// The launch uses programmatic dependent launch, so back-to-back decode calls overlap their launch
+// latency and prologue with the previous call's tail.
 #include "common.cuh"
 #include "launch.h"
 
@@ -25,7 +27,7 @@ constexpr int kDecThreads = 128;
 constexpr int kDecWarps = 4;
 constexpr int kTile = 64;          // tokens per pipeline stage
 constexpr int kStages = 3;
-constexpr int kMaxChunk = 2048;    // tokens per work item (index staging buffer)
+constexpr int kMaxChunk = 2048;    // tokens per work item in the two-kernel mode
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -39,46 +41,14 @@ struct DecParams {
   const int32_t* cu_k;
   const int32_t* cu_nloc;
   const int32_t* local_idx;
-  float* part_o;     // [max_items][Hkv][G][D]   unnormalised
-  float* part_ml;    // [max_items][Hkv][G][2]   (m in log2 units, l)
   uint16_t* out;
   float* lse;
   int32_t* dev_status;
   int64_t ts, hs;
-  int32_t B, Hq, Hkv, G, K_tot, NL_tot, chunk;
-  int32_t csize;     // fused mode: CTAs per (sequence, KV head) = cluster size
+  int32_t B, Hq, Hkv, G, K_tot, NL_tot;
+  int32_t csize;     // CTAs per (sequence, KV head) = cluster size
   float scale_log2;
 };
-
-// Work item -> (sequence b, chunk c within b, first item of b).  Computed redundantly per warp.
-__device__ __forceinline__ bool find_item(const DecParams& p, int item, int lane, int& b_out, int& c_out) {
-  int acc = 0;
-  for (int b0 = 0; b0 < p.B; b0 += 32) {
-    const int b = b0 + lane;
-    int nch = 0;
-    if (b < p.B) {
-      const int n = (p.cu_k[b + 1] - p.cu_k[b]) + (p.cu_nloc[b + 1] - p.cu_nloc[b]);
-      nch = (n + p.chunk - 1) / p.chunk;
-    }
-    int inc = nch;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, inc, off);
-      if (lane >= off) inc += v;
-    }
-    const int tot = __shfl_sync(0xffffffffu, inc, 31);
-    if (item < acc + tot) {
-      const unsigned hit = __ballot_sync(0xffffffffu, item < acc + inc);
-      const int src = __ffs(hit) - 1;
-      const int exc = __shfl_sync(0xffffffffu, inc - nch, src);
-      b_out = b0 + src;
-      c_out = item - (acc + exc);
-      return true;
-    }
-    acc += tot;
-  }
-  return false;
-}
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -122,8 +92,7 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // kHi: the KV head has more than 8 query rows, so MMA rows 8..15 carry data too.
-// kFused: the CTAs of a (sequence, KV head) form a cluster and merge their partials through DSMEM.
-template <int D, bool kHi, bool kFused>
+template <int D, bool kHi>
 __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const DecParams p) {
   constexpr int kRowBytes = D * 2;
   constexpr int kChunksPerRow = D / 8;                       // 16-byte chunks
@@ -132,25 +101,20 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* sk = smem_raw;                                    // [kStages][kTile][D] bf16, swizzled
   uint8_t* sv = smem_raw + kStages * kTileBytes;
-  int32_t* s_idx = reinterpret_cast<int32_t*>(smem_raw + 2 * kStages * kTileBytes);   // [kMaxChunk]
+  uint8_t* s_valid = smem_raw + 2 * kStages * kTileBytes;    // [kStages][kTile] 1 = row holds a real token
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
   pdl_launch_dependents();
   pdl_wait();
-  int b, c;
-  if (kFused) {
-    b = blockIdx.z;
-    c = blockIdx.x;                                            // rank in the cluster
-  } else if (!find_item(p, blockIdx.x, lane, b, c)) {
-    return;
-  }
+  const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
+  const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
   const int kb = p.cu_k[b + 1] - p.cu_k[b];
   const int nl = p.cu_nloc[b + 1] - p.cu_nloc[b];
   const int c0 = p.cu[b];
   const int nseq = p.cu[b + 1] - c0;
   // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
-  const int span = kFused ? ((((kb + nl + p.csize - 1) / p.csize) + kTile - 1) / kTile) * kTile : p.chunk;
+  const int span = ((((kb + nl + p.csize - 1) / p.csize) + kTile - 1) / kTile) * kTile;
   const int range_beg = min(kb + nl, c * span);
   const int range_end = min(kb + nl, range_beg + span);
 
@@ -160,14 +124,25 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   const uint16_t* lv_base = p.local_v + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
   const uint32_t sk_u32 = smem_u32(sk), sv_u32 = smem_u32(sv);
 
-  int pos_beg = 0, ntok = 0;                                   // current sub-chunk (at most kMaxChunk tokens)
-  auto load_tile = [&](int tile, int stage) {
+  const int pos_beg = range_beg, ntok = range_end - range_beg;
+  const int ntiles = (ntok + kTile - 1) / kTile;
+  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] - kb;   // indexed by list position
+  // Local indices of the rows this thread copies in `tile` (read one tile ahead of their use).
+  auto fetch_idx = [&](int tile, int (&idx)[kCopiesPerThread]) {
+#pragma unroll
+    for (int i = 0; i < kCopiesPerThread; ++i) {
+      const int li = tile * kTile + (tid + i * kDecThreads) / kChunksPerRow;
+      const int pos = pos_beg + li;
+      idx[i] = (li < ntok && pos >= kb) ? __ldg(idx_base + pos) : 0;
+    }
+  };
+  auto load_tile = [&](int tile, int stage, const int (&idx)[kCopiesPerThread]) {
 #pragma unroll
     for (int i = 0; i < kCopiesPerThread; ++i) {
       const int qid = tid + i * kDecThreads;
       const int row = qid / kChunksPerRow;
       const int col = qid % kChunksPerRow;
-      const int li = tile * kTile + row;                      // index within the chunk
+      const int li = tile * kTile + row;                      // index within this CTA's range
       const int pos = pos_beg + li;
       const uint16_t* srck = p.packed_k;
       const uint16_t* srcv = p.packed_v;
@@ -178,17 +153,20 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
           srcv = pv_base + (int64_t)pos * D + col * 8;
           bytes = 16;
         } else {
-          const int t = s_idx[li];
-          if (t >= 0) {
+          const int t = idx[i];
+          if (t >= 0 && t < nseq) {
             srck = lk_base + (int64_t)t * p.ts + col * 8;
             srcv = lv_base + (int64_t)t * p.ts + col * 8;
             bytes = 16;
+          } else if (col == 0) {
+            raise(p.dev_status, SG_ERR_INDEX);
           }
         }
       }
       const uint32_t off = stage * kTileBytes + row * kRowBytes + ((col ^ (row & 7)) << 4);
-      cp_async16(sk_u32 + off, srck, bytes);
+      cp_async16(sk_u32 + off, srck, bytes);                  // bytes == 0 zero-fills the row
       cp_async16(sv_u32 + off, srcv, bytes);
+      if (col == 0) s_valid[stage * kTile + row] = bytes ? 1 : 0;
     }
   };
 
@@ -212,25 +190,17 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   for (int i = 0; i < D / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
-#pragma unroll 1
-  for (pos_beg = range_beg; pos_beg < range_end; pos_beg += kMaxChunk) {
-  ntok = min(range_end - pos_beg, kMaxChunk);
-  const int ntiles = (ntok + kTile - 1) / kTile;
-  // Stage this sub-chunk's local indices (validated); packed positions get 0.
-  for (int i = tid; i < ntok; i += kDecThreads) {
-    const int pos = pos_beg + i;
-    int v = 0;
-    if (pos >= kb) {
-      v = __ldg(p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + (pos - kb));
-      if (v < 0 || v >= nseq) { v = -1; raise(p.dev_status, SG_ERR_INDEX); }
-    }
-    s_idx[i] = v;
-  }
-  __syncthreads();
+  int idx_next[kCopiesPerThread];
+  {
+    int idx_pro[kStages - 1][kCopiesPerThread];
 #pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) {
-    if (s < ntiles) load_tile(s, s);
-    cp_async_commit();
+    for (int s = 0; s < kStages - 1; ++s) fetch_idx(s, idx_pro[s]);
+    fetch_idx(kStages - 1, idx_next);
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) {
+      if (s < ntiles) load_tile(s, s, idx_pro[s]);
+      cp_async_commit();
+    }
   }
 
 #pragma unroll 1
@@ -239,8 +209,9 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     __syncthreads();
     {
       const int nt = tile + kStages - 1;
-      if (nt < ntiles) load_tile(nt, nt % kStages);
+      if (nt < ntiles) load_tile(nt, nt % kStages, idx_next);
       cp_async_commit();
+      fetch_idx(nt + 1, idx_next);
     }
     const int stage = tile % kStages;
     const uint32_t k_st = sk_u32 + stage * kTileBytes;
@@ -268,8 +239,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     for (int j = 0; j < 2; ++j) {
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const int li = tile * kTile + wrow + j * 8 + 2 * (lane & 3) + e;
-        const bool valid = li < ntok && s_idx[li] >= 0;
+        const bool valid = s_valid[stage * kTile + wrow + j * 8 + 2 * (lane & 3) + e] != 0;
         s_acc[j][e] = valid ? s_acc[j][e] * p.scale_log2 : -INFINITY;
         mx_lo = fmaxf(mx_lo, s_acc[j][e]);
         if (kHi) {
@@ -340,7 +310,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   }
   cp_async_wait<0>();
   __syncthreads();
-  }  // sub-chunks
 
   // merge the four warps through shared memory (the pipeline buffers are free now)
   float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
@@ -361,9 +330,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   float* sm_co = sm_l + kDecWarps * 16;                       // CTA-level partial: O [16][D], m [16], l [16]
   float* sm_cm = sm_co + 16 * D;
   float* sm_cl = sm_cm + 16;
-  const int64_t slot = (int64_t)blockIdx.x * p.Hkv + g;
-  float* po = p.part_o + slot * p.G * D;
-  float* pml = p.part_ml + slot * p.G * 2;
   for (int e = tid; e < p.G * D; e += kDecThreads) {
     const int r = e / D, col = e - r * D;
     float M = -INFINITY;
@@ -377,15 +343,10 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
       L += sm_l[w * 16 + r] * f;
       O += sm_o[(w * 16 + r) * D + col] * f;
     }
-    if (kFused) {
-      sm_co[e] = O;
-      if (col == 0) { sm_cm[r] = M; sm_cl[r] = L; }
-    } else {
-      po[e] = O;
-      if (col == 0) { pml[2 * r] = M; pml[2 * r + 1] = L; }
-    }
+    sm_co[e] = O;
+    if (col == 0) { sm_cm[r] = M; sm_cl[r] = L; }
   }
-  if (kFused) {
+  {
     // Every CTA of the cluster merges a slice of the G*D outputs, reading all ranks' partials.
     const int cs = p.csize;
     if (cs > 1) cluster_sync_all(); else __syncthreads();
@@ -394,15 +355,26 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
     for (int e = e_beg + tid; e < e_end; e += kDecThreads) {
       const int r = e / D, col = e - r * D;
+      float mj[8], lj[8], oj[8];                             // all ranks' partials, loaded independently
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        mj[j] = -INFINITY; lj[j] = 0.f; oj[j] = 0.f;
+        if (j < cs) {
+          mj[j] = cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r];
+          lj[j] = cs > 1 ? ld_dsmem_f32(sm_cl + r, j) : sm_cl[r];
+          oj[j] = cs > 1 ? ld_dsmem_f32(sm_co + e, j) : sm_co[e];
+        }
+      }
       float M = -INFINITY;
-      for (int j = 0; j < cs; ++j) M = fmaxf(M, cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) M = fmaxf(M, mj[j]);
       const float Mu = M == -INFINITY ? 0.f : M;
       float L = 0.f, O = 0.f;
-      for (int j = 0; j < cs; ++j) {
-        const float mj = cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r];
-        const float f = exp2f(mj - Mu);
-        L += (cs > 1 ? ld_dsmem_f32(sm_cl + r, j) : sm_cl[r]) * f;
-        O += (cs > 1 ? ld_dsmem_f32(sm_co + e, j) : sm_co[e]) * f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float f = exp2f(mj[j] - Mu);
+        L += lj[j] * f;
+        O += oj[j] * f;
       }
       outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
       if (p.lse && col == 0) p.lse[(int64_t)b * p.Hq + (int64_t)g * p.G + r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
@@ -411,69 +383,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   }
 }
 
-// Merge the per-chunk partials of one (sequence, query head): m = max m_j, l = sum l_j 2^(m_j-m),
-// o = sum o_j 2^(m_j-m) / l.  One block of D threads per (h, b).
 template <int D>
-__global__ void __launch_bounds__(D) decode_combine_kernel(const DecParams p) {
-  __shared__ int s_part[D / 32];
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  pdl_launch_dependents();
-  pdl_wait();
-  const int g = h / p.G, r = h - g * p.G;
-  // first work item of sequence b = number of chunks of the sequences before it
-  int cnt = 0;
-  for (int bb = tid; bb < b; bb += D) {
-    const int n = (p.cu_k[bb + 1] - p.cu_k[bb]) + (p.cu_nloc[bb + 1] - p.cu_nloc[bb]);
-    cnt += (n + p.chunk - 1) / p.chunk;
-  }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-  if ((tid & 31) == 0) s_part[tid >> 5] = cnt;
-  __syncthreads();
-  int first = 0;
-#pragma unroll
-  for (int w = 0; w < D / 32; ++w) first += s_part[w];
-  const int n = (p.cu_k[b + 1] - p.cu_k[b]) + (p.cu_nloc[b + 1] - p.cu_nloc[b]);
-  const int nch = (n + p.chunk - 1) / p.chunk;
-
-  float M = -INFINITY;
-  for (int c = 0; c < nch; ++c) M = fmaxf(M, p.part_ml[(((int64_t)(first + c) * p.Hkv + g) * p.G + r) * 2]);
-  const float Mu = M == -INFINITY ? 0.f : M;
-  float L = 0.f, O = 0.f;
-  for (int c = 0; c < nch; ++c) {
-    const int64_t slot = (int64_t)(first + c) * p.Hkv + g;
-    const float f = exp2f(p.part_ml[(slot * p.G + r) * 2] - Mu);
-    L += p.part_ml[(slot * p.G + r) * 2 + 1] * f;
-    O += p.part_o[(slot * p.G + r) * D + tid] * f;
-  }
-  const float res = L > 0.f ? O / L : 0.f;
-  reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)b * p.Hq + h) * D + tid] = __float2bfloat16_rn(res);
-  if (p.lse && tid == 0) p.lse[(int64_t)b * p.Hq + h] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
-}
-
-template <int D>
-constexpr int decode_smem_bytes() { return 2 * kStages * kTile * D * 2 + kMaxChunk * 4; }
+constexpr int decode_smem_bytes() { return 2 * kStages * kTile * D * 2 + kStages * kTile; }
 
 }  // namespace
 
-int decode_chunk_tokens(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
-  const int64_t total = (int64_t)total_sel + total_loc;
-  const int target_items = (4 * kNumSMs + shape->num_kv_heads - 1) / shape->num_kv_heads;   // ~4 CTAs per SM
-  int64_t chunk = (total + target_items - 1) / target_items;
-  chunk = ((chunk + kTile - 1) / kTile) * kTile;
-  if (chunk < kTile) chunk = kTile;
-  if (chunk > kMaxChunk) chunk = kMaxChunk;
-  return (int)chunk;
-}
-
-// Fused (cluster) mode: CTAs per (sequence, KV head), a power of two <= 8; 0 selects the two-kernel mode.
-// The fused mode is used unless there are too few (sequence, head) pairs to fill the GPU with clusters of
-// 8 while each list is long enough to feed many more CTAs.
+// CTAs per (sequence, KV head) = cluster size: a power of two <= 8 (the portable cluster limit).
 int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
   const int64_t pairs = (int64_t)shape->batch * shape->num_kv_heads;
-  if (shape->batch > 65535) return 0;
   const int64_t avg_tiles = (((int64_t)total_sel + total_loc) / shape->batch + kTile - 1) / kTile;
-  if (pairs * 8 < kNumSMs && avg_tiles >= 64) return 0;
   int by_work = 1;
   while (by_work < 8 && by_work * 2 * 2 <= avg_tiles) by_work *= 2;        // at least two tiles per CTA
   int by_fill = 1;
@@ -481,18 +399,7 @@ int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_
   return by_work < by_fill ? by_work : by_fill;
 }
 
-static int64_t decode_max_items(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
-  const int chunk = decode_chunk_tokens(shape, total_sel, total_loc);
-  return ((int64_t)total_sel + total_loc + chunk - 1) / chunk + shape->batch;
-}
-
-size_t decode_workspace_bytes(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
-  if (shape->num_kv_heads < 1 || shape->num_q_heads < 1 || shape->batch < 1) return 0;
-  if (decode_cluster_size(shape, total_sel, total_loc) > 0) return 0;       // fused mode keeps partials on chip
-  const int64_t items = decode_max_items(shape, total_sel, total_loc);
-  const int G = shape->num_q_heads / shape->num_kv_heads;
-  return (size_t)items * shape->num_kv_heads * G * (shape->head_dim + 2) * sizeof(float);
-}
+size_t decode_workspace_bytes(const sg_shape*, int32_t, int32_t) { return 0; }   // partials stay on chip
 
 }  // namespace sg
 
@@ -514,10 +421,9 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
       !aligned16(workspace) || (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)))
     return SG_ERR_INVALID;
   if (!(softmax_scale >= 0.f)) return SG_ERR_INVALID;
+  (void)workspace_bytes;                                      // no workspace is needed: partials stay on chip
   const int D = shape->head_dim;
   const int G = shape->num_q_heads / shape->num_kv_heads;
-  const int64_t items = decode_max_items(shape, total_sel, total_loc);
-  if (items > 0x7fffffffLL || shape->num_kv_heads > 65535 || shape->batch > 65535) return SG_ERR_UNSUPPORTED;
   DecParams p;
   p.q = static_cast<const uint16_t*>(q);
   p.packed_k = static_cast<const uint16_t*>(packed_k ? packed_k : q);
@@ -527,9 +433,7 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.cu = shape->cu_seqlens;
   p.cu_k = cu_k;
   p.cu_nloc = cu_nloc;
-  p.local_idx = local_idx;
-  p.part_o = nullptr;
-  p.part_ml = nullptr;
+  p.local_idx = local_idx ? local_idx : cu_nloc;
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.dev_status = dev_status;
@@ -541,56 +445,33 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.G = G;
   p.K_tot = total_sel;
   p.NL_tot = total_loc;
-  p.chunk = decode_chunk_tokens(shape, total_sel, total_loc);
-  p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
-
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   p.csize = decode_cluster_size(shape, total_sel, total_loc);
-  const bool fused = p.csize > 0;
+  p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
+  const int64_t grid_x = (int64_t)shape->batch * p.csize;
+  if (grid_x > 0x7fffffffLL || shape->num_kv_heads > 65535) return SG_ERR_UNSUPPORTED;
 
   cudaLaunchAttribute attrs[2];
   attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attrs[0].val.programmaticStreamSerializationAllowed = 1;
   attrs[1].id = cudaLaunchAttributeClusterDimension;
-  attrs[1].val.clusterDim.x = fused ? (unsigned)p.csize : 1u;
+  attrs[1].val.clusterDim.x = (unsigned)p.csize;
   attrs[1].val.clusterDim.y = 1;
   attrs[1].val.clusterDim.z = 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.stream = s;
+  cfg.stream = static_cast<cudaStream_t>(stream);
   cfg.attrs = attrs;
+  cfg.numAttrs = p.csize > 1 ? 2 : 1;
   cfg.blockDim = dim3(kDecThreads);
-#define SG_LAUNCH_DECODE(DD, HI, FU)                                                                  \
-  do {                                                                                                \
-    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI, FU>), decode_smem_bytes<DD>());                     \
-    cfg.dynamicSmemBytes = decode_smem_bytes<DD>();                                                   \
-    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<DD, HI, FU>, p));                      \
+  // one launch: sequences with empty lists still get out = 0 and lse = -inf
+  cfg.gridDim = dim3((unsigned)grid_x, (unsigned)shape->num_kv_heads);
+#define SG_LAUNCH_DECODE(DD, HI)                                                          \
+  do {                                                                                    \
+    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI>), decode_smem_bytes<DD>());             \
+    cfg.dynamicSmemBytes = decode_smem_bytes<DD>();                                       \
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<DD, HI>, p));              \
   } while (0)
-#define SG_LAUNCH_DECODE_D(DD)                                                                        \
-  do {                                                                                                \
-    if (fused) { if (G > 8) SG_LAUNCH_DECODE(DD, true, true); else SG_LAUNCH_DECODE(DD, false, true); } \
-    else       { if (G > 8) SG_LAUNCH_DECODE(DD, true, false); else SG_LAUNCH_DECODE(DD, false, false); } \
-  } while (0)
-  if (fused) {
-    // one launch: grid (cluster size, H_kv, B); sequences with empty lists still get out = 0, lse = -inf
-    cfg.gridDim = dim3((unsigned)p.csize, (unsigned)shape->num_kv_heads, (unsigned)shape->batch);
-    cfg.numAttrs = p.csize > 1 ? 2 : 1;
-    if (D == 128) SG_LAUNCH_DECODE_D(128); else SG_LAUNCH_DECODE_D(64);
-    return SG_OK;
-  }
-  const size_t need = decode_workspace_bytes(shape, total_sel, total_loc);
-  if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
-  p.part_o = static_cast<float*>(workspace);
-  p.part_ml = p.part_o + items * shape->num_kv_heads * G * D;
-  cfg.numAttrs = 1;
-  if (total_sel + total_loc > 0) {
-    cfg.gridDim = dim3((unsigned)items, (unsigned)shape->num_kv_heads);
-    if (D == 128) SG_LAUNCH_DECODE_D(128); else SG_LAUNCH_DECODE_D(64);
-  }
-#undef SG_LAUNCH_DECODE_D
+  if (D == 128) { if (G > 8) SG_LAUNCH_DECODE(128, true); else SG_LAUNCH_DECODE(128, false); }
+  else          { if (G > 8) SG_LAUNCH_DECODE(64, true);  else SG_LAUNCH_DECODE(64, false); }
 #undef SG_LAUNCH_DECODE
-  cfg.gridDim = dim3((unsigned)shape->num_q_heads, (unsigned)shape->batch);
-  cfg.dynamicSmemBytes = 0;
-  if (D == 128) { cfg.blockDim = dim3(128); SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<128>, p)); }
-  else          { cfg.blockDim = dim3(64);  SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<64>, p)); }
   return SG_OK;
 }

@@ -8,8 +8,6 @@
 namespace sg {
 size_t score_workspace_bytes(const sg_shape* shape);
 size_t decode_workspace_bytes(const sg_shape* shape, int32_t total_sel, int32_t total_loc);
-// Tokens per split-KV work item chosen for a decode call of this size (a multiple of 64).
-int decode_chunk_tokens(const sg_shape* shape, int32_t total_sel, int32_t total_loc);
-// Cluster size of the fused decode mode for this call, or 0 when the two-kernel mode is used.
+// Cluster size (CTAs per sequence and KV head) the decode kernel uses for a call of this size.
 int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_loc);
 }  // namespace sg

@@ -43,14 +43,18 @@ def test_host_side_argument_checks_need_no_gpu():
     bad = ctypes.c_void_p(0x1004)        # misaligned
     assert lib.sg_pack_kv(ctypes.byref(s), bad, fake, fake, fake, 4, fake, fake, None, None) == sg.SG_ERR_INVALID
     assert lib.sg_pack_kv(ctypes.byref(s), fake, fake, fake, fake, -1, fake, fake, None, None) == sg.SG_ERR_INVALID
-    # decode, long lists on few heads (the two-kernel mode): workspace too small is reported before any launch
+    # decode: split-KV partials are merged on chip (cluster mode), no workspace is ever needed
+    s = sg.Shape(1, 1, 8, 2, 128, 4, 16384, 16384, 0x1000, 16384 * 256, 256, 128)
+    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 8192, 4096) == 0
+    assert sg.sg_workspace_bytes(sg.SG_OP_PACK_KV, s, 4, 4) == 0
     lib.sg_sparse_decode_attn.restype = ctypes.c_int
     lib.sg_sparse_decode_attn.argtypes = sg._lib.sg_sparse_decode_attn.argtypes
-    s = sg.Shape(1, 1, 8, 2, 128, 4, 16384, 16384, 0x1000, 16384 * 256, 256, 128)
-    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 8192, 4096) > 16
-    rc = lib.sg_sparse_decode_attn(ctypes.byref(s), fake, fake, fake, fake, 8192, fake, fake, fake, fake, 4096, 0.0,
-                                   fake, None, fake, 16, None, None)
-    assert rc == sg.SG_ERR_WORKSPACE
-    # short lists are merged on chip (cluster mode) and need no workspace
-    assert sg.sg_workspace_bytes(sg.SG_OP_SPARSE_DECODE_ATTN, s, 64, 64) == 0
-    assert sg.sg_workspace_bytes(sg.SG_OP_PACK_KV, s, 4, 4) == 0
+    s2 = sg.Shape(2, 1, 8, 2, 128, 4, 16384, 16384, 0x1000, 16384 * 256, 256, 128)     # decode takes one layer per call
+    rc = lib.sg_sparse_decode_attn(ctypes.byref(s2), fake, fake, fake, fake, 64, fake, fake, fake, fake, 64, 0.0,
+                                   fake, None, None, 0, None, None)
+    assert rc == sg.SG_ERR_INVALID
+    # score: workspace too small is reported before any launch
+    lib.sg_score.restype = ctypes.c_int
+    lib.sg_score.argtypes = sg._lib.sg_score.argtypes
+    assert sg.sg_workspace_bytes(sg.SG_OP_SCORE, s) > 16
+    assert lib.sg_score(ctypes.byref(s), fake, fake, fake, fake, 16, None, None) == sg.SG_ERR_WORKSPACE
