@@ -106,7 +106,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
   pdl_launch_dependents();
-  pdl_wait();
   const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
   const int kb = p.cu_k[b + 1] - p.cu_k[b];
@@ -170,21 +169,6 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     }
   };
 
-  // Q fragments (A operand, 16 x D, rows >= G are zero).
-  const int r_lo = lane >> 2, r_hi = r_lo + 8;
-  uint32_t qa[D / 16][4];
-  {
-    const uint16_t* qb = p.q + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
-#pragma unroll
-    for (int kk = 0; kk < D / 16; ++kk) {
-      const int col = kk * 16 + 2 * (lane & 3);
-      qa[kk][0] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col) : 0u;
-      qa[kk][2] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col + 8) : 0u;
-      qa[kk][1] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col) : 0u;
-      qa[kk][3] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col + 8) : 0u;
-    }
-  }
-
   float o_acc[D / 8][4];
 #pragma unroll
   for (int i = 0; i < D / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
@@ -200,6 +184,24 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     for (int s = 0; s < kStages - 1; ++s) {
       if (s < ntiles) load_tile(s, s, idx_pro[s]);
       cp_async_commit();
+    }
+  }
+
+  // Everything above reads only the KV sources, the index lists and the prefix arrays, which are stable
+  // inputs of a decode step; q (and the outputs) are ordered after all earlier work in the stream.
+  pdl_wait();
+  // Q fragments (A operand, 16 x D, rows >= G are zero).
+  const int r_lo = lane >> 2, r_hi = r_lo + 8;
+  uint32_t qa[D / 16][4];
+  {
+    const uint16_t* qb = p.q + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
+#pragma unroll
+    for (int kk = 0; kk < D / 16; ++kk) {
+      const int col = kk * 16 + 2 * (lane & 3);
+      qa[kk][0] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col) : 0u;
+      qa[kk][2] = r_lo < p.G ? *reinterpret_cast<const uint32_t*>(qb + r_lo * D + col + 8) : 0u;
+      qa[kk][1] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col) : 0u;
+      qa[kk][3] = (kHi && r_hi < p.G) ? *reinterpret_cast<const uint32_t*>(qb + r_hi * D + col + 8) : 0u;
     }
   }
 
