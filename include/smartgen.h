@@ -174,8 +174,9 @@ sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void
  *   - The call allocates nothing and frees nothing.  The first call on each device looks up the
  *     array's device address (one cudaGetSymbolAddress with that device current); make that first
  *     call before starting any stream capture on the device.
- *   - All calls on a device share the one array, which keeps the previous call's contents.  Nothing
- *     in it needs clearing (every slot is written before it is read within a call), but two calls
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  The
+ *     call itself clears the few counters in it that must start at zero (a memset on `stream`);
+ *     everything else is written before it is read within a call.  But two calls
  *     that overlap on the GPU -- different streams, or one stream's call still running when another
  *     starts -- race on it and give undefined importance.  Serialise them, or use sg_score with
  *     separate workspaces.

@@ -12,14 +12,19 @@
 //          each epilogue thread owns one key (one TMEM lane) and adds exp2(s*c - lse_r) over the
 //          query-row columns; lse_r is a per-column constant read from shared memory.
 //
-// Both passes share one warp-specialised skeleton: warp 0 feeds 128-key K tiles (and Q once) with
-// TMA into 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM
-// accumulator stages, warps 2-9 (two per TMEM lane quarter, each taking half of the columns)
-// drain them with tcgen05.ld.  The score matrix never leaves the SM.  Per-chunk row statistics
-// (pass 1) go to a small workspace; pass 2 merges them in its prologue.
+// One persistent kernel runs both passes: warp 0 feeds Q and 128-key K tiles with TMA into
+// 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM accumulator
+// stages, warps 2-9 (two per TMEM lane quarter, each taking half of the columns) drain them with
+// tcgen05.ld.  The score matrix never leaves the SM.  Work items (a pass, a layer/KV head, a chunk of
+// key tiles of one sequence) are laid out so that pass 2 of a (layer, KV head) unit follows its pass 1
+// by a lag of a few units: close enough that the unit's keys are still in L2 for the second read
+// (K crosses HBM once), far enough that the statistics pass 2 needs are already published.  Pass 1
+// items publish per-chunk row statistics to a small workspace and bump a per-unit counter; pass 2 items
+// wait (bounded) on that counter.  A pass-2 item only depends on items at smaller schedule positions and
+// pass-1 items never wait, so the schedule cannot deadlock for any grid size.
 //
-// Every mbarrier wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word,
-// stops issuing work, drains its own TMA copies with bounded waits, frees its TMEM and returns.
+// Every wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word, stops issuing
+// work, drains its own TMA copies with bounded waits, frees its TMEM and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -40,12 +45,15 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct ScoreParams {
   const int32_t* cu;
   float* importance;
-  float* part_m;           // [L][Hkv][max_items][Ralloc]
+  int* p1_done;            // [U] pass-1 items finished per unit (zeroed by the host call)
+  float* part_m;           // [U][max_items][Ralloc] per-item row statistics (log2 domain max, sum)
   float* part_l;
   int32_t* dev_status;
   int64_t T;
   int32_t B, Hkv, G, W, R, Rpad, Ralloc;
-  int32_t tiles_per_chunk, max_items, k_stages;
+  int32_t U;               // units = layers x KV heads
+  int32_t lag;             // pass 2 of unit u is scheduled `lag` units after its pass 1
+  int32_t tiles_per_chunk, max_items, k_stages, q_bufs;
   float scale_log2;
 };
 
@@ -177,7 +185,69 @@ __device__ __forceinline__ bool find_chunk(const ScoreParams& p, int item, int l
   return false;
 }
 
-template <int D, bool kPass1>
+// Position in the persistent schedule -> work item.  The schedule is a sequence of slots; slot s holds the
+// pass-2 items of unit (s - lag) followed by the pass-1 items of unit s, a unit being one (layer, KV head)
+// with all its sequences (C items per pass).  CTA k walks positions k, k + grid, k + 2*grid, ...  A pass-2
+// item depends only on pass-1 items at smaller positions, and pass-1 items never wait, so the item at the
+// smallest unfinished position can always run: the schedule cannot deadlock whatever the grid size.
+struct ScoreItem {
+  int pass;          // 1 or 2; 0 = no item at this position
+  int unit, l, g, b;
+  int tile_beg, tile_end;
+  int item_in_unit;  // this item's index among the unit's C items (its partial-statistics slot)
+  int first_item_b;  // index of sequence b's first item in the unit
+  int nch_b;         // number of items (chunks) of sequence b
+};
+
+// Number of items per unit and pass: sum over sequences of ceil(tiles / tiles_per_chunk).  Warp-collective.
+__device__ __forceinline__ int items_per_unit(const ScoreParams& p, int lane) {
+  int acc = 0;
+  for (int b0 = 0; b0 < p.B; b0 += 32) {
+    const int b = b0 + lane;
+    int nch = 0;
+    if (b < p.B) {
+      const int tiles = (p.cu[b + 1] - p.cu[b] + kTileKeys - 1) / kTileKeys;
+      nch = (tiles + p.tiles_per_chunk - 1) / p.tiles_per_chunk;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) nch += __shfl_xor_sync(0xffffffffu, nch, off);
+    acc += nch;
+  }
+  return acc;
+}
+
+// Warp-collective: every lane gets the same item.
+__device__ __forceinline__ ScoreItem decode_position(const ScoreParams& p, long long pos, int C, int lane) {
+  ScoreItem it;
+  it.pass = 0;
+  const int slot = (int)(pos / (2 * C));
+  const int r = (int)(pos - (long long)slot * (2 * C));
+  int unit, j;
+  if (r < C) { unit = slot - p.lag; j = r; it.pass = 2; } else { unit = slot; j = r - C; it.pass = 1; }
+  if (unit < 0 || unit >= p.U) { it.pass = 0; return it; }
+  it.unit = unit;
+  it.l = unit / p.Hkv;
+  it.g = unit - it.l * p.Hkv;
+  it.item_in_unit = j;
+  int b, chunk, first, nch;
+  if (!find_chunk(p, j, lane, b, chunk, first, nch)) { it.pass = 0; return it; }
+  it.b = b;
+  it.first_item_b = first;
+  it.nch_b = nch;
+  const int N = p.cu[b + 1] - p.cu[b];
+  const int tiles_total = (N + kTileKeys - 1) / kTileKeys;
+  it.tile_beg = chunk * p.tiles_per_chunk;
+  it.tile_end = min(tiles_total, it.tile_beg + p.tiles_per_chunk);
+  return it;
+}
+
+__device__ __forceinline__ int ld_acquire_gpu(const int* ptr) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
   constexpr int kSub = D / 64;                        // 64-element (128-byte) sub-tiles along d
@@ -186,35 +256,26 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const int q_sub_bytes = p.Ralloc * 128;
-  uint8_t* q_smem = smem;
-  uint8_t* k_smem = q_smem + kSub * q_sub_bytes;
+  const int q_buf_bytes = kSub * q_sub_bytes;
+  uint8_t* q_smem = smem;                                            // [q_bufs] Q operands
+  uint8_t* k_smem = q_smem + p.q_bufs * q_buf_bytes;                  // [k_stages] K tiles
   uint8_t* tail = k_smem + p.k_stages * kKStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 1 + 4*4 barriers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 17 * 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 17 * 8 + 4);
-  float* sm_f = reinterpret_cast<float*>(tail + 160);         // pass 1: m[2][Ralloc], l[2][Ralloc]; pass 2: lse2[Ralloc], part[2][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 4 Q + 4*4 ring barriers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 20 * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 20 * 8 + 4);
+  float* sm_f = reinterpret_cast<float*>(tail + 176);                 // pass 1: m[2][Ralloc], l[2][Ralloc]; pass 2: lse2[Ralloc], part[2][128]
 
-  const uint32_t bar_q = smem_u32(&bars[0]);
-  auto bar_kfull = [&](int s) { return smem_u32(&bars[1 + s]); };
-  auto bar_kempty = [&](int s) { return smem_u32(&bars[1 + kMaxKStages + s]); };
-  auto bar_afull = [&](int s) { return smem_u32(&bars[1 + 2 * kMaxKStages + s]); };
-  auto bar_aempty = [&](int s) { return smem_u32(&bars[1 + 2 * kMaxKStages + kAccStages + s]); };
+  auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
+  auto bar_qempty = [&](int s) { return smem_u32(&bars[2 + s]); };
+  auto bar_kfull = [&](int s) { return smem_u32(&bars[4 + s]); };
+  auto bar_kempty = [&](int s) { return smem_u32(&bars[4 + kMaxKStages + s]); };
+  auto bar_afull = [&](int s) { return smem_u32(&bars[4 + 2 * kMaxKStages + s]); };
+  auto bar_aempty = [&](int s) { return smem_u32(&bars[4 + 2 * kMaxKStages + kAccStages + s]); };
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = blockIdx.y, l = blockIdx.z;
-  int b, chunk, first_item, nch;
-  if (!find_chunk(p, blockIdx.x, lane, b, chunk, first_item, nch)) return;
-  const int c0 = p.cu[b];
-  const int N = p.cu[b + 1] - c0;
-  const int Weff = min(p.W, N);
-  const int tiles_total = (N + kTileKeys - 1) / kTileKeys;
-  const int tile_beg = chunk * p.tiles_per_chunk;
-  const int tile_end = min(tiles_total, tile_beg + p.tiles_per_chunk);
-  const int nblk = kPass1 ? (p.R + 127) / 128 : (p.Rpad + 127) / 128;
-  const int first_win = N - Weff;                     // position of window row 0; keys <= it are visible to all rows
 
   if (tid == 0) {
-    mbar_init(bar_q, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), 1); }
     for (int s = 0; s < kMaxKStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
     for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), kEpiThreads / 32); }
     *abort_flag = 0;
@@ -226,13 +287,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     tmem_relinquish();
   }
   if (p.R < p.Ralloc) {
-    // Rows R..Ralloc-1 of the Q operand are never written by TMA: zero them so that padded MMA rows/columns
-    // are finite.  (The 128-byte swizzle only permutes 16-byte chunks inside a row's own 128 bytes.)
+    // Rows R..Ralloc-1 of the Q operands are never written by TMA: zero them once so that padded MMA
+    // rows/columns are finite.  (The 128-byte swizzle only permutes 16-byte chunks inside a row's own 128 bytes.)
     const int words = (p.Ralloc - p.R) * 32;
-    for (int dc = 0; dc < kSub; ++dc) {
-      uint32_t* z = reinterpret_cast<uint32_t*>(q_smem + dc * q_sub_bytes + p.R * 128);
-      for (int i = tid; i < words; i += kScoreThreads) z[i] = 0u;
-    }
+    for (int qb = 0; qb < p.q_bufs; ++qb)
+      for (int dc = 0; dc < kSub; ++dc) {
+        uint32_t* z = reinterpret_cast<uint32_t*>(q_smem + qb * q_buf_bytes + dc * q_sub_bytes + p.R * 128);
+        for (int i = tid; i < words; i += kScoreThreads) z[i] = 0u;
+      }
     fence_proxy_async();
   }
   tc_fence_before();
@@ -240,80 +302,105 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  const int C = items_per_unit(p, lane);                               // same value in every thread
+  const long long npos = (long long)(p.U + p.lag) * 2 * C;
+
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      mbar_arrive_expect_tx(bar_q, (uint32_t)(kSub * p.G * p.W * 128));
+    // ------------------------------------------------------------ TMA producer (lane 0 issues)
+    int stage = 0, n_item = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
+      const ScoreItem it = decode_position(p, pos, C, lane);
+      if (it.pass == 0) continue;
+      if (lane == 0) {
+        const int qb = n_item % p.q_bufs;
+        const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
+        ok = mbar_wait(bar_qempty(qb), qph ^ 1u, abort_flag);
+        if (ok) {
+          mbar_arrive_expect_tx(bar_qfull(qb), (uint32_t)(kSub * p.G * p.W * 128));
 #pragma unroll
-      for (int dc = 0; dc < kSub; ++dc)
-        tma_load_4d(smem_u32(q_smem + dc * q_sub_bytes), &tmap_q, bar_q, dc * 64, g * p.G, 0, l * p.B + b);
-      int stage = 0, issued = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
-        ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
+          for (int dc = 0; dc < kSub; ++dc)
+            tma_load_4d(smem_u32(q_smem + qb * q_buf_bytes + dc * q_sub_bytes), &tmap_q, bar_qfull(qb), dc * 64, it.g * p.G, 0,
+                        it.l * p.B + it.b);
+          const int c0 = p.cu[it.b];
+          for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
+            ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
 #pragma unroll
-        for (int dc = 0; dc < kSub; ++dc)
-          tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, g,
-                      c0 + tile * kTileKeys, l);
-        ++issued;
-        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
-      }
-      // Wait until the MMAs have released every stage: after this no arrival on a K barrier is pending.
-      for (int i = 0; i < p.k_stages && ok; ++i) {
-        ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
-        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
-      }
-      if (!ok) {
-        // Drain: wait (bounded) until every copy this thread issued has landed, so none is in flight at exit.
-        volatile int never = 0;
-        mbar_wait(bar_q, 0, &never);
-        for (int i = 0; i < issued; ++i) {
-          const int s = i % p.k_stages;
-          const uint32_t ph = (uint32_t)((i / p.k_stages) & 1);
-          if (i + p.k_stages >= issued) mbar_wait(bar_kfull(s), ph, &never);
+            for (int dc = 0; dc < kSub; ++dc)
+              tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, it.g,
+                          c0 + tile * kTileKeys, it.l);
+            if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
+          }
         }
+      }
+      ++n_item;
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    }
+    if (lane == 0) {
+      // Wait until the MMAs have released every K stage and Q buffer, so that no barrier arrival and no copy
+      // of this CTA is still pending when it exits.  (On an aborted run the waits give up after their limit.)
+      volatile int never = 0;
+      for (int i = 0; i < p.k_stages; ++i) {
+        if (!mbar_wait(bar_kempty(stage), phase ^ 1u, ok ? abort_flag : &never)) break;
+        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
+      }
+      for (int i = 0; i < p.q_bufs; ++i) {
+        const int n = n_item + i;
+        if (!mbar_wait(bar_qempty(n % p.q_bufs), (uint32_t)(((n / p.q_bufs) & 1) ^ 1), ok ? abort_flag : &never)) break;
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      bool ok = mbar_wait(bar_q, 0, abort_flag);
-      tc_fence_after();
-      int ks = 0, as = 0;
-      uint32_t kph = 0, aph = 0;
-      const uint32_t q_addr = smem_u32(q_smem);
-      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
-        ok = mbar_wait(bar_kfull(ks), kph, abort_flag);
-        if (!ok) break;
+    // ------------------------------------------------------------ MMA issuer (lane 0 issues)
+    int ks = 0, as = 0, n_item = 0;
+    uint32_t kph = 0, aph = 0;
+    bool ok = true;
+    for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
+      const ScoreItem it = decode_position(p, pos, C, lane);
+      if (it.pass == 0) continue;
+      if (lane == 0) {
+        const int qb = n_item % p.q_bufs;
+        const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
+        ok = mbar_wait(bar_qfull(qb), qph, abort_flag);
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
-        for (int blk = 0; blk < nblk && ok; ++blk) {
-          ok = mbar_wait(bar_aempty(as), aph ^ 1u, abort_flag);
+        const bool pass1 = it.pass == 1;
+        const int nblk = pass1 ? (p.R + 127) / 128 : (p.Rpad + 127) / 128;
+        const uint32_t q_addr = smem_u32(q_smem + qb * q_buf_bytes);
+        for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
+          ok = mbar_wait(bar_kfull(ks), kph, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const int ncols = kPass1 ? 128 : min(128, p.Rpad - blk * 128);
-          const uint32_t idesc = make_idesc(128, ncols);
-          const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
+          const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
+          for (int blk = 0; blk < nblk && ok; ++blk) {
+            ok = mbar_wait(bar_aempty(as), aph ^ 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int ncols = pass1 ? 128 : min(128, p.Rpad - blk * 128);
+            const uint32_t idesc = make_idesc(128, ncols);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
 #pragma unroll
-          for (int dc = 0; dc < kSub; ++dc) {
-            const uint32_t qa = q_addr + dc * q_sub_bytes + blk * (128 * 128);
-            const uint32_t ka = k_addr + dc * kKSubBytes;
+            for (int dc = 0; dc < kSub; ++dc) {
+              const uint32_t qa = q_addr + dc * q_sub_bytes + blk * (128 * 128);
+              const uint32_t ka = k_addr + dc * kKSubBytes;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              const uint64_t dq = smem_desc_sw128(qa + kk * 32);
-              const uint64_t dk = smem_desc_sw128(ka + kk * 32);
-              umma_bf16(d_tmem, kPass1 ? dq : dk, kPass1 ? dk : dq, idesc, (dc | kk) != 0 ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk) {
+                const uint64_t dq = smem_desc_sw128(qa + kk * 32);
+                const uint64_t dk = smem_desc_sw128(ka + kk * 32);
+                umma_bf16(d_tmem, pass1 ? dq : dk, pass1 ? dk : dq, idesc, (dc | kk) != 0 ? 1u : 0u);
+              }
             }
+            umma_commit(bar_afull(as));
+            if (++as == kAccStages) { as = 0; aph ^= 1u; }
           }
-          umma_commit(bar_afull(as));
-          if (++as == kAccStages) { as = 0; aph ^= 1u; }
+          if (ok) umma_commit(bar_kempty(ks));
+          if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
         }
-        if (ok) umma_commit(bar_kempty(ks));
-        if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
+        if (ok) umma_commit(bar_qempty(qb));
       }
+      ++n_item;
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
@@ -322,65 +409,72 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     const int lane_grp = warp & 3;                     // TMEM lane quarter this warp may access
     const int row_in_tile = lane_grp * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
-    const size_t part_base = (((size_t)l * p.Hkv + g) * p.max_items) * p.Ralloc;
     int as = 0;
     uint32_t aph = 0;
     bool ok = true;
+    for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every warp meets the named barriers
+      const ScoreItem it = decode_position(p, pos, C, lane);
+      if (it.pass == 0) continue;
+      const int c0 = p.cu[it.b];
+      const int N = p.cu[it.b + 1] - c0;
+      const int Weff = min(p.W, N);
+      const int first_win = N - Weff;                  // position of window row 0; keys <= it are visible to all rows
+      const size_t part_base = (size_t)it.unit * p.max_items * p.Ralloc;
 
-    if (kPass1) {
-      float* sm_m = sm_f;                              // [2][Ralloc]
-      float* sm_l = sm_f + 2 * p.Ralloc;
-      for (int r = etid; r < 2 * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
-      epi_bar_sync();
-      for (int tile = tile_beg; tile < tile_end && ok; ++tile) {
-        const int t0 = tile * kTileKeys;
-        const bool all_visible = t0 + kTileKeys - 1 <= first_win;
-        for (int blk = 0; blk < nblk && ok; ++blk) {
-          ok = mbar_wait(bar_afull(as), aph, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const int r = blk * 128 + row_in_tile;
-          const bool row_ok = r < p.R && (r / p.G) < Weff;
-          const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
-          float m = sm_m[half * p.Ralloc + r], lsum = sm_l[half * p.Ralloc + r];
+      if (it.pass == 1) {
+        const int nblk = (p.R + 127) / 128;
+        float* sm_m = sm_f;                            // [2][Ralloc]
+        float* sm_l = sm_f + 2 * p.Ralloc;
+        for (int r = etid; r < 2 * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
+        epi_bar_sync();
+        for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
+          const int t0 = tile * kTileKeys;
+          const bool all_visible = t0 + kTileKeys - 1 <= first_win;
+          for (int blk = 0; blk < nblk && ok; ++blk) {
+            ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int r = blk * 128 + row_in_tile;
+            const bool row_ok = r < p.R && (r / p.G) < Weff;
+            const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
+            float m = sm_m[half * p.Ralloc + r], lsum = sm_l[half * p.Ralloc + r];
 #pragma unroll 1
-          for (int j = 0; j < 2; ++j) {
-            const int col0 = half * 64 + j * 32;
-            float v[32];
-            tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
-            if (all_visible && row_ok) {
-              float mx = v[0];
+            for (int j = 0; j < 2; ++j) {
+              const int col0 = half * 64 + j * 32;
+              float v[32];
+              tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
+              if (all_visible && row_ok) {
+                float mx = v[0];
 #pragma unroll
-              for (int c = 1; c < 32; ++c) mx = fmaxf(mx, v[c]);
-              const float mn = fmaxf(m, mx * p.scale_log2);
-              float s = 0.f;
+                for (int c = 1; c < 32; ++c) mx = fmaxf(mx, v[c]);
+                const float mn = fmaxf(m, mx * p.scale_log2);
+                float s = 0.f;
 #pragma unroll
-              for (int c = 0; c < 32; ++c) s += exp2f(fmaf(v[c], p.scale_log2, -mn));
-              lsum = lsum * exp2f(m - mn) + s;
-              m = mn;
-            } else if (col0 <= cmax) {
-              float mx = -INFINITY;
+                for (int c = 0; c < 32; ++c) s += exp2f(fmaf(v[c], p.scale_log2, -mn));
+                lsum = lsum * exp2f(m - mn) + s;
+                m = mn;
+              } else if (col0 <= cmax) {
+                float mx = -INFINITY;
 #pragma unroll
-              for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, v[c]) : mx;
-              const float mn = fmaxf(m, mx * p.scale_log2);
-              float s = 0.f;
+                for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, v[c]) : mx;
+                const float mn = fmaxf(m, mx * p.scale_log2);
+                float s = 0.f;
 #pragma unroll
-              for (int c = 0; c < 32; ++c) s += (col0 + c <= cmax) ? exp2f(fmaf(v[c], p.scale_log2, -mn)) : 0.f;
-              lsum = lsum * exp2f(m - mn) + s;
-              m = mn;
+                for (int c = 0; c < 32; ++c) s += (col0 + c <= cmax) ? exp2f(fmaf(v[c], p.scale_log2, -mn)) : 0.f;
+                lsum = lsum * exp2f(m - mn) + s;
+                m = mn;
+              }
             }
+            sm_m[half * p.Ralloc + r] = m;
+            sm_l[half * p.Ralloc + r] = lsum;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_aempty(as));
+            if (++as == kAccStages) { as = 0; aph ^= 1u; }
           }
-          sm_m[half * p.Ralloc + r] = m;
-          sm_l[half * p.Ralloc + r] = lsum;
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_aempty(as));
-          if (++as == kAccStages) { as = 0; aph ^= 1u; }
         }
-      }
-      epi_bar_sync();
-      if (ok && !*abort_flag) {
-        const size_t slot = part_base + (size_t)blockIdx.x * p.Ralloc;
+        epi_bar_sync();
+        const size_t slot = part_base + (size_t)it.item_in_unit * p.Ralloc;
         for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
           const float m0 = sm_m[r], m1 = sm_m[p.Ralloc + r];
           const float M = fmaxf(m0, m1);
@@ -388,69 +482,90 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           p.part_m[slot + r] = M;
           p.part_l[slot + r] = sm_l[r] * exp2f(m0 - Mu) + sm_l[p.Ralloc + r] * exp2f(m1 - Mu);
         }
-      }
-    } else {
-      float* lse2 = sm_f;                              // [Ralloc]
-      float* sm_part = sm_f + p.Ralloc;                // [2][128]
-      for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
-        float val = INFINITY;                          // rows outside the window: exp2(x - inf) = 0
-        if (r < p.R && (r / p.G) < Weff) {
-          float M = -INFINITY;
-          for (int c = 0; c < nch; ++c) M = fmaxf(M, p.part_m[part_base + (size_t)(first_item + c) * p.Ralloc + r]);
-          float L = 0.f;
-          for (int c = 0; c < nch; ++c) {
-            const size_t o = part_base + (size_t)(first_item + c) * p.Ralloc + r;
-            L += p.part_l[o] * exp2f(p.part_m[o] - M);
+        __threadfence();                               // this thread's statistics are visible GPU-wide ...
+        epi_bar_sync();
+        if (etid == 0 && ok && !*abort_flag) atomicAdd(p.p1_done + it.unit, 1);   // ... before the item is counted as done
+      } else {
+        const int nblk = (p.Rpad + 127) / 128;
+        float* lse2 = sm_f;                            // [Ralloc]
+        float* sm_part = sm_f + p.Ralloc;              // [2][128]
+        // Wait (bounded) until every pass-1 item of this unit has published its row statistics.
+        if (etid == 0 && ok) {
+          uint64_t t0 = 0;
+          for (uint32_t spin = 0;; ++spin) {
+            if (ld_acquire_gpu(p.p1_done + it.unit) >= C) break;
+            if (*abort_flag) break;
+            if ((spin & 63u) == 63u) {
+              const uint64_t now = global_timer_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > 2000000000ull) { *abort_flag = 1; break; }
+            }
+            __nanosleep(64);
           }
-          val = M + log2f(L);
         }
-        lse2[r] = val;
-      }
-      epi_bar_sync();
-      for (int tile = tile_beg; tile < tile_end; ++tile) {   // no early exit: every warp meets the named barrier
-        const int t = tile * kTileKeys + row_in_tile;  // this thread's key
-        const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
-        const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
-        float acc = 0.f;
-        for (int blk = 0; blk < nblk && ok; ++blk) {
-          ok = mbar_wait(bar_afull(as), aph, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const int ncols = min(128, p.Rpad - blk * 128);
+        epi_bar_sync();
+        if (*abort_flag) ok = false;
+        for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
+          float val = INFINITY;                        // rows outside the window: exp2(x - inf) = 0
+          if (ok && r < p.R && (r / p.G) < Weff) {
+            float M = -INFINITY;
+            for (int c = 0; c < it.nch_b; ++c) M = fmaxf(M, __ldcg(p.part_m + part_base + (size_t)(it.first_item_b + c) * p.Ralloc + r));
+            float L = 0.f;
+            for (int c = 0; c < it.nch_b; ++c) {
+              const size_t o = part_base + (size_t)(it.first_item_b + c) * p.Ralloc + r;
+              L += __ldcg(p.part_l + o) * exp2f(__ldcg(p.part_m + o) - M);
+            }
+            val = M + log2f(L);
+          }
+          lse2[r] = val;
+        }
+        epi_bar_sync();
+        for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
+          const int t = tile * kTileKeys + row_in_tile;  // this thread's key
+          const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
+          const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
+          float acc = 0.f;
+          for (int blk = 0; blk < nblk && ok; ++blk) {
+            ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int ncols = min(128, p.Rpad - blk * 128);
 #pragma unroll 1
-          for (int j = 0; j < 2; ++j) {
-            const int col0 = half * 64 + j * 32;
-            if (col0 >= ncols) break;
-            float v[32];
-            tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
-            const float* ls = lse2 + blk * 128 + col0;
-            if (all_visible && col0 + 32 <= ncols) {
+            for (int j = 0; j < 2; ++j) {
+              const int col0 = half * 64 + j * 32;
+              if (col0 >= ncols) break;
+              float v[32];
+              tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
+              const float* ls = lse2 + blk * 128 + col0;
+              if (all_visible && col0 + 32 <= ncols) {
 #pragma unroll
-              for (int c = 0; c < 32; c += 4) {
-                const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                acc += exp2f(fmaf(v[c], p.scale_log2, -l4.x));
-                acc += exp2f(fmaf(v[c + 1], p.scale_log2, -l4.y));
-                acc += exp2f(fmaf(v[c + 2], p.scale_log2, -l4.z));
-                acc += exp2f(fmaf(v[c + 3], p.scale_log2, -l4.w));
-              }
-            } else {
+                for (int c = 0; c < 32; c += 4) {
+                  const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                  acc += exp2f(fmaf(v[c], p.scale_log2, -l4.x));
+                  acc += exp2f(fmaf(v[c + 1], p.scale_log2, -l4.y));
+                  acc += exp2f(fmaf(v[c + 2], p.scale_log2, -l4.z));
+                  acc += exp2f(fmaf(v[c + 3], p.scale_log2, -l4.w));
+                }
+              } else {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
-                acc += vis ? exp2f(fmaf(v[c], p.scale_log2, -ls[c])) : 0.f;
+                for (int c = 0; c < 32; ++c) {
+                  const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
+                  acc += vis ? exp2f(fmaf(v[c], p.scale_log2, -ls[c])) : 0.f;
+                }
               }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_aempty(as));
+            if (++as == kAccStages) { as = 0; aph ^= 1u; }
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_aempty(as));
-          if (++as == kAccStages) { as = 0; aph ^= 1u; }
+          float* part = sm_part + (tile & 1) * 128;
+          if (half == 1) part[row_in_tile] = acc;
+          epi_bar_sync();
+          if (half == 0 && ok && t < N)
+            p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + c0 + t] = acc + part[row_in_tile];
         }
-        float* part = sm_part + (tile & 1) * 128;
-        if (half == 1) part[row_in_tile] = acc;
-        epi_bar_sync();
-        if (half == 0 && ok && t < N)
-          p.importance[((size_t)l * p.Hkv + g) * p.T + c0 + t] = acc + part[row_in_tile];
+        epi_bar_sync();                                // lse2 / part are reused by the next item
       }
     }
   }
@@ -482,7 +597,8 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 struct ScorePlan {
-  int R, Rpad, Ralloc, k_stages, tiles_per_chunk, max_items, smem_bytes;
+  int R, Rpad, Ralloc, k_stages, q_bufs, tiles_per_chunk, max_items, smem_bytes, U, lag;
+  size_t counter_bytes, workspace_bytes;
   bool ok;
 };
 
@@ -495,30 +611,43 @@ ScorePlan plan_score(const sg_shape* s) {
   pl.Ralloc = (pl.R + 127) & ~127;
   const int q_bytes = pl.Ralloc * D * 2;
   const int k_stage = kTileKeys * D * 2;
-  const int tail = 160 + 4 * pl.Ralloc * 4 + 2 * 128 * 4;
-  const int avail = kSmemLimit - 1024 - q_bytes - tail;
-  pl.k_stages = avail / k_stage;
+  const int tail = 176 + 4 * pl.Ralloc * 4 + 2 * 128 * 4;
+  const int avail = kSmemLimit - 1024 - tail;
+  // Two Q buffers let the next item's queries load while the current item computes; fall back to one
+  // when that would leave fewer than three K stages.
+  pl.q_bufs = 2;
+  pl.k_stages = (avail - 2 * q_bytes) / k_stage;
+  if (pl.k_stages < 3) { pl.q_bufs = 1; pl.k_stages = (avail - q_bytes) / k_stage; }
   if (pl.k_stages > kMaxKStages) pl.k_stages = kMaxKStages;
   pl.ok = pl.k_stages >= 2 && s->window <= 256 && pl.R <= 1024;
-  pl.smem_bytes = 1024 + q_bytes + pl.k_stages * k_stage + tail;
+  pl.smem_bytes = 1024 + pl.q_bufs * q_bytes + pl.k_stages * k_stage + tail;
   if (pl.smem_bytes < 120 * 1024) pl.smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes the whole TMEM
-  // chunking of the key axis: about four waves of CTAs over the SMs, 4..32 tiles per chunk
-  const int64_t total_tiles = ((int64_t)s->total_tokens / kTileKeys + s->batch) * s->num_kv_heads * s->num_layers;
-  int64_t tpc = total_tiles / (4 * kNumSMs);
-  if (tpc < 4) tpc = 4;
-  if (tpc > 32) tpc = 32;
-  pl.tiles_per_chunk = (int)tpc;
-  const int64_t max_tiles = (int64_t)s->total_tokens / kTileKeys + s->batch;
-  pl.max_items = (int)(max_tiles / pl.tiles_per_chunk + s->batch);
+  pl.U = s->num_layers * s->num_kv_heads;
+  // chunking of the key axis: 8 tiles per item, halved while that leaves fewer than ~6 items per SM and pass
+  const int64_t tiles_per_unit = (int64_t)s->total_tokens / kTileKeys + s->batch;
+  int tpc = 8;
+  while (tpc > 4 && (tiles_per_unit / tpc + s->batch) * pl.U < 6 * kNumSMs) tpc /= 2;
+  pl.tiles_per_chunk = tpc;
+  pl.max_items = (int)(tiles_per_unit / tpc + s->batch + 1);
+  // Pass 2 of a unit trails its pass 1 by `lag` units.  The lag must span more schedule positions than there
+  // are CTAs (each slot holds about 2*C positions), otherwise pass-2 items run in the same wave as the pass-1
+  // items they wait for and stall; beyond that it is kept as small as possible so that the unit's keys are
+  // still in L2 for the second read.
+  const int64_t c_est = (tiles_per_unit - s->batch) / tpc + 1;
+  int64_t lag = (5 * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
+  if (lag > pl.U) lag = pl.U;
+  pl.lag = (int)lag;
+  pl.counter_bytes = ((size_t)pl.U * sizeof(int) + 255) & ~(size_t)255;
+  pl.workspace_bytes = pl.counter_bytes + (size_t)2 * pl.U * pl.max_items * pl.Ralloc * sizeof(float);
   return pl;
 }
 
 }  // namespace
 
 size_t score_workspace_bytes(const sg_shape* s) {
-  if (s->num_kv_heads < 1 || s->num_q_heads < 1 || s->window < 1) return 0;
-  const ScorePlan pl = plan_score(s);
-  return (size_t)2 * s->num_layers * s->num_kv_heads * pl.max_items * pl.Ralloc * sizeof(float);
+  if (s->num_kv_heads < 1 || s->num_q_heads < 1 || s->window < 1 || s->num_layers < 1) return 0;
+  if (s->num_q_heads % s->num_kv_heads != 0) return 0;
+  return plan_score(s).workspace_bytes;
 }
 
 }  // namespace sg
@@ -533,7 +662,6 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   if (!aligned16(q_win) || !aligned16(k_cache) || !aligned16(importance) || !aligned16(workspace)) return SG_ERR_INVALID;
   const ScorePlan pl = plan_score(shape);
   if (!pl.ok) return SG_ERR_UNSUPPORTED;
-  if (shape->num_kv_heads > 65535 || shape->num_layers > 65535) return SG_ERR_UNSUPPORTED;
   const size_t need = score_workspace_bytes(shape);
   if (!workspace || workspace_bytes < need) return SG_ERR_WORKSPACE;
   EncodeTiledFn encode = encode_tiled_fn();
@@ -574,8 +702,9 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   ScoreParams p;
   p.cu = shape->cu_seqlens;
   p.importance = importance;
-  p.part_m = static_cast<float*>(workspace);
-  p.part_l = p.part_m + (size_t)shape->num_layers * shape->num_kv_heads * pl.max_items * pl.Ralloc;
+  p.p1_done = static_cast<int*>(workspace);
+  p.part_m = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
+  p.part_l = p.part_m + (size_t)pl.U * pl.max_items * pl.Ralloc;
   p.dev_status = dev_status;
   p.T = shape->total_tokens;
   p.B = shape->batch;
@@ -585,22 +714,30 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   p.R = pl.R;
   p.Rpad = pl.Rpad;
   p.Ralloc = pl.Ralloc;
+  p.U = pl.U;
+  p.lag = pl.lag;
   p.tiles_per_chunk = pl.tiles_per_chunk;
   p.max_items = pl.max_items;
   p.k_stages = pl.k_stages;
+  p.q_bufs = pl.q_bufs;
   p.scale_log2 = kLog2e / sqrtf((float)D);
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const dim3 grid((unsigned)pl.max_items, (unsigned)shape->num_kv_heads, (unsigned)shape->num_layers);
-#define SG_LAUNCH_SCORE(DD, P1)                                                                                      \
-  do {                                                                                                               \
-    SG_ENSURE_SMEM((score_kernel<DD, P1>), pl.smem_bytes);                                                           \
-    score_kernel<DD, P1><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);                               \
-    SG_CUDA_TRY(cudaGetLastError());                                                                                 \
-  } while (0)
-  if (D == 128) { SG_LAUNCH_SCORE(128, true); SG_LAUNCH_SCORE(128, false); }
-  else          { SG_LAUNCH_SCORE(64, true);  SG_LAUNCH_SCORE(64, false); }
-#undef SG_LAUNCH_SCORE
+  // the per-unit completion counters must start at zero on every call (also on every graph replay)
+  SG_CUDA_TRY(cudaMemsetAsync(workspace, 0, pl.counter_bytes, s));
+  int dev = 0, sms = kNumSMs;
+  SG_CUDA_TRY(cudaGetDevice(&dev));
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = kNumSMs;
+  const long long max_pos = (long long)(pl.U + pl.lag) * 2 * pl.max_items;
+  const unsigned grid = (unsigned)(max_pos < sms ? max_pos : sms);     // persistent: one CTA per SM
+  if (D == 128) {
+    SG_ENSURE_SMEM((score_kernel<128>), pl.smem_bytes);
+    score_kernel<128><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);
+  } else {
+    SG_ENSURE_SMEM((score_kernel<64>), pl.smem_bytes);
+    score_kernel<64><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);
+  }
+  SG_CUDA_TRY(cudaGetLastError());
   return SG_OK;
 }
 
