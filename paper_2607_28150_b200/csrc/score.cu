@@ -14,13 +14,13 @@
 //
 // One persistent kernel runs both passes: warp 0 feeds Q and 128-key K tiles with TMA into
 // 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM accumulator
-// stages, warps 2-9 (two per TMEM lane quarter, each taking half of the columns) drain them with
+// stages (a ring of two per epilogue warpgroup), warps 2-9 (two warpgroups, each owning alternate key tiles) drain them with pipelined
 // tcgen05.ld.  The score matrix never leaves the SM.  Work items (a pass, a layer/KV head, a chunk of
 // key tiles of one sequence) are laid out so that pass 2 of a (layer, KV head) unit follows its pass 1
 // by a lag of a few units: close enough that the unit's keys are still in L2 for the second read
 // (K crosses HBM once), far enough that the statistics pass 2 needs are already published.  Pass 1
 // items publish per-chunk row statistics to a small workspace and bump a per-unit counter; pass 2 items
-// wait (bounded) on that counter.  A pass-2 item only depends on items at smaller schedule positions and
+// wait (bounded) on that counter and merge the chunks' statistics into the rows' log-sum-exps.  A pass-2 item only depends on items at smaller schedule positions and
 // pass-1 items never wait, so the schedule cannot deadlock for any grid size.
 //
 // Every wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word, stops issuing
@@ -120,8 +120,9 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
-  uint32_t r[32];
+// Asynchronous TMEM load of 32 consecutive fp32 columns of this thread's lane.  The registers may only be
+// read after tmem_wait_ld() on the same array.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t (&r)[32], uint32_t taddr) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -131,9 +132,16 @@ __device__ __forceinline__ void tmem_ld32(float (&v)[32], uint32_t taddr) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Wait for this thread's outstanding TMEM loads.  The array is passed in/out so that every later use of its
+// registers depends on this statement.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
 }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
@@ -153,38 +161,6 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Work item -> (sequence, chunk of key tiles); also returns the sequence's first item.
-__device__ __forceinline__ bool find_chunk(const ScoreParams& p, int item, int lane, int& b_out, int& c_out, int& first_out, int& nch_out) {
-  int acc = 0;
-  for (int b0 = 0; b0 < p.B; b0 += 32) {
-    const int b = b0 + lane;
-    int nch = 0;
-    if (b < p.B) {
-      const int tiles = (p.cu[b + 1] - p.cu[b] + kTileKeys - 1) / kTileKeys;
-      nch = (tiles + p.tiles_per_chunk - 1) / p.tiles_per_chunk;
-    }
-    int inc = nch;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, inc, off);
-      if (lane >= off) inc += v;
-    }
-    const int tot = __shfl_sync(0xffffffffu, inc, 31);
-    if (item < acc + tot) {
-      const unsigned hit = __ballot_sync(0xffffffffu, item < acc + inc);
-      const int src = __ffs(hit) - 1;
-      const int exc = __shfl_sync(0xffffffffu, inc - nch, src);
-      b_out = b0 + src;
-      first_out = acc + exc;
-      c_out = item - first_out;
-      nch_out = __shfl_sync(0xffffffffu, nch, src);
-      return true;
-    }
-    acc += tot;
-  }
-  return false;
-}
-
 // Position in the persistent schedule -> work item.  The schedule is a sequence of slots; slot s holds the
 // pass-2 items of unit (s - lag) followed by the pass-1 items of unit s, a unit being one (layer, KV head)
 // with all its sequences (C items per pass).  CTA k walks positions k, k + grid, k + 2*grid, ...  A pass-2
@@ -193,33 +169,18 @@ __device__ __forceinline__ bool find_chunk(const ScoreParams& p, int item, int l
 struct ScoreItem {
   int pass;          // 1 or 2; 0 = no item at this position
   int unit, l, g, b;
+  int c0, N;         // first token and length of sequence b
   int tile_beg, tile_end;
   int item_in_unit;  // this item's index among the unit's C items (its partial-statistics slot)
   int first_item_b;  // index of sequence b's first item in the unit
   int nch_b;         // number of items (chunks) of sequence b
 };
 
-// Number of items per unit and pass: sum over sequences of ceil(tiles / tiles_per_chunk).  Warp-collective.
-__device__ __forceinline__ int items_per_unit(const ScoreParams& p, int lane) {
-  int acc = 0;
-  for (int b0 = 0; b0 < p.B; b0 += 32) {
-    const int b = b0 + lane;
-    int nch = 0;
-    if (b < p.B) {
-      const int tiles = (p.cu[b + 1] - p.cu[b] + kTileKeys - 1) / kTileKeys;
-      nch = (tiles + p.tiles_per_chunk - 1) / p.tiles_per_chunk;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) nch += __shfl_xor_sync(0xffffffffu, nch, off);
-    acc += nch;
-  }
-  return acc;
-}
-
-// Warp-collective: every lane gets the same item.
-__device__ __forceinline__ ScoreItem decode_position(const ScoreParams& p, long long pos, int C, int lane) {
+// s_cu[b] = cu_seqlens[b]; s_prefix[b] = number of items of the sequences before b (s_prefix[B] = C).
+__device__ __forceinline__ ScoreItem decode_position(const ScoreParams& p, long long pos, const int* s_cu, const int* s_prefix) {
   ScoreItem it;
   it.pass = 0;
+  const int C = s_prefix[p.B];
   const int slot = (int)(pos / (2 * C));
   const int r = (int)(pos - (long long)slot * (2 * C));
   int unit, j;
@@ -229,14 +190,18 @@ __device__ __forceinline__ ScoreItem decode_position(const ScoreParams& p, long 
   it.l = unit / p.Hkv;
   it.g = unit - it.l * p.Hkv;
   it.item_in_unit = j;
-  int b, chunk, first, nch;
-  if (!find_chunk(p, j, lane, b, chunk, first, nch)) { it.pass = 0; return it; }
-  it.b = b;
-  it.first_item_b = first;
-  it.nch_b = nch;
-  const int N = p.cu[b + 1] - p.cu[b];
-  const int tiles_total = (N + kTileKeys - 1) / kTileKeys;
-  it.tile_beg = chunk * p.tiles_per_chunk;
+  int lo = 0, hi = p.B;                                  // largest b with s_prefix[b] <= j
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (s_prefix[mid] <= j) lo = mid; else hi = mid;
+  }
+  it.b = lo;
+  it.first_item_b = s_prefix[lo];
+  it.nch_b = s_prefix[lo + 1] - it.first_item_b;
+  it.c0 = s_cu[lo];
+  it.N = s_cu[lo + 1] - it.c0;
+  const int tiles_total = (it.N + kTileKeys - 1) / kTileKeys;
+  it.tile_beg = (j - it.first_item_b) * p.tiles_per_chunk;
   it.tile_end = min(tiles_total, it.tile_beg + p.tiles_per_chunk);
   return it;
 }
@@ -246,7 +211,6 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* ptr) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
   return v;
 }
-
 template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
@@ -260,24 +224,29 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   uint8_t* q_smem = smem;                                            // [q_bufs] Q operands
   uint8_t* k_smem = q_smem + p.q_bufs * q_buf_bytes;                  // [k_stages] K tiles
   uint8_t* tail = k_smem + p.k_stages * kKStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 4 Q + 4*4 ring barriers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 20 * 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 20 * 8 + 4);
-  float* sm_f = reinterpret_cast<float*>(tail + 176);                 // pass 1: m[2][Ralloc], l[2][Ralloc]; pass 2: lse2[Ralloc], part[2][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 20 barriers (28 slots reserved)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 28 * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 28 * 8 + 4);
+  float* lse_buf = reinterpret_cast<float*>(tail + 240);              // [Ralloc] row log-sum-exps of the current pass-2 item
+  float* sm_stat = lse_buf + p.Ralloc;                            // pass 1: m[2][Ralloc], l[2][Ralloc]
+  int* s_cu = reinterpret_cast<int*>(sm_stat + 4 * p.Ralloc);         // [B+1]
+  int* s_prefix = s_cu + p.B + 1;                                     // [B+1]
 
   auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
   auto bar_qempty = [&](int s) { return smem_u32(&bars[2 + s]); };
   auto bar_kfull = [&](int s) { return smem_u32(&bars[4 + s]); };
-  auto bar_kempty = [&](int s) { return smem_u32(&bars[4 + kMaxKStages + s]); };
-  auto bar_afull = [&](int s) { return smem_u32(&bars[4 + 2 * kMaxKStages + s]); };
-  auto bar_aempty = [&](int s) { return smem_u32(&bars[4 + 2 * kMaxKStages + kAccStages + s]); };
+  auto bar_kempty = [&](int s) { return smem_u32(&bars[8 + s]); };
+  auto bar_afull = [&](int s) { return smem_u32(&bars[12 + s]); };
+  auto bar_aempty = [&](int s) { return smem_u32(&bars[16 + s]); };
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), 1);
+    }
     for (int s = 0; s < kMaxKStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
-    for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), kEpiThreads / 32); }
+    for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), 4); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -285,6 +254,28 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
+  }
+  if (warp == 2) {
+    // sequence offsets and the per-sequence item prefix, once per CTA
+    int acc = 0;
+    for (int b0 = 0; b0 <= p.B; b0 += 32) {
+      const int b = b0 + lane;
+      int nch = 0;
+      if (b <= p.B) s_cu[b] = p.cu[b];
+      if (b < p.B) {
+        const int tiles = (p.cu[b + 1] - p.cu[b] + kTileKeys - 1) / kTileKeys;
+        nch = (tiles + p.tiles_per_chunk - 1) / p.tiles_per_chunk;
+      }
+      int inc = nch;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += v;
+      }
+      if (b < p.B) s_prefix[b + 1] = acc + inc;
+      acc += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) s_prefix[0] = 0;
   }
   if (p.R < p.Ralloc) {
     // Rows R..Ralloc-1 of the Q operands are never written by TMA: zero them once so that padded MMA
@@ -301,48 +292,43 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-
-  const int C = items_per_unit(p, lane);                               // same value in every thread
+  const int C = s_prefix[p.B];
   const long long npos = (long long)(p.U + p.lag) * 2 * C;
+  volatile int never = 0;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (lane 0 issues)
-    int stage = 0, n_item = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
-      const ScoreItem it = decode_position(p, pos, C, lane);
-      if (it.pass == 0) continue;
-      if (lane == 0) {
+    // ------------------------------------------------------------ TMA producer (one thread)
+    if (lane == 0) {
+      int stage = 0, n_item = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
+        const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
+        if (it.pass == 0) continue;
         const int qb = n_item % p.q_bufs;
         const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
+        ++n_item;
         ok = mbar_wait(bar_qempty(qb), qph ^ 1u, abort_flag);
-        if (ok) {
-          mbar_arrive_expect_tx(bar_qfull(qb), (uint32_t)(kSub * p.G * p.W * 128));
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_qfull(qb), (uint32_t)(kSub * p.G * p.W * 128));
+#pragma unroll
+        for (int dc = 0; dc < kSub; ++dc)
+          tma_load_4d(smem_u32(q_smem + qb * q_buf_bytes + dc * q_sub_bytes), &tmap_q, bar_qfull(qb), dc * 64, it.g * p.G, 0,
+                      it.l * p.B + it.b);
+        for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
+          ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
 #pragma unroll
           for (int dc = 0; dc < kSub; ++dc)
-            tma_load_4d(smem_u32(q_smem + qb * q_buf_bytes + dc * q_sub_bytes), &tmap_q, bar_qfull(qb), dc * 64, it.g * p.G, 0,
-                        it.l * p.B + it.b);
-          const int c0 = p.cu[it.b];
-          for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
-            ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
-            if (!ok) break;
-            mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
-#pragma unroll
-            for (int dc = 0; dc < kSub; ++dc)
-              tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, it.g,
-                          c0 + tile * kTileKeys, it.l);
-            if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
-          }
+            tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, it.g,
+                        it.c0 + tile * kTileKeys, it.l);
+          if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
         }
       }
-      ++n_item;
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    }
-    if (lane == 0) {
-      // Wait until the MMAs have released every K stage and Q buffer, so that no barrier arrival and no copy
-      // of this CTA is still pending when it exits.  (On an aborted run the waits give up after their limit.)
-      volatile int never = 0;
+      // Wait until the MMAs have released every K stage and Q buffer, so that
+      // no barrier arrival and no copy of this CTA is still pending when it exits.  (On an aborted run the
+      // waits give up after their limit.)
       for (int i = 0; i < p.k_stages; ++i) {
         if (!mbar_wait(bar_kempty(stage), phase ^ 1u, ok ? abort_flag : &never)) break;
         if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
@@ -353,17 +339,23 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (lane 0 issues)
-    int ks = 0, as = 0, n_item = 0;
-    uint32_t kph = 0, aph = 0;
-    bool ok = true;
-    for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
-      const ScoreItem it = decode_position(p, pos, C, lane);
-      if (it.pass == 0) continue;
-      if (lane == 0) {
+    // ------------------------------------------------------------ MMA issuer (one thread)
+    // Accumulator stages 0-1 feed epilogue warpgroup 0, stages 2-3 warpgroup 1; a key tile goes to the
+    // warpgroup given by the parity of the CTA's running tile count.  Each ring is consumed by one warpgroup
+    // only, so no waiter ever falls more than one mbarrier phase behind.
+    if (lane == 0) {
+      int ks = 0, n_item = 0;
+      int ring0 = 0, ring1 = 0;
+      uint32_t kph = 0, rph0 = 0, rph1 = 0, tile_count = 0;
+      bool ok = true;
+      for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
+        const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
+        if (it.pass == 0) continue;
         const int qb = n_item % p.q_bufs;
         const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
+        ++n_item;
         ok = mbar_wait(bar_qfull(qb), qph, abort_flag);
+        if (!ok) break;
         tc_fence_after();
         const bool pass1 = it.pass == 1;
         const int nblk = pass1 ? (p.R + 127) / 128 : (p.Rpad + 127) / 128;
@@ -373,8 +365,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           if (!ok) break;
           tc_fence_after();
           const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
+          const bool odd = ((tile_count++) & 1u) != 0;
           for (int blk = 0; blk < nblk && ok; ++blk) {
-            ok = mbar_wait(bar_aempty(as), aph ^ 1u, abort_flag);
+            const int as = odd ? 2 + ring1 : ring0;
+            ok = mbar_wait(bar_aempty(as), (odd ? rph1 : rph0) ^ 1u, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const int ncols = pass1 ? 128 : min(128, p.Rpad - blk * 128);
@@ -382,99 +376,118 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
 #pragma unroll
             for (int dc = 0; dc < kSub; ++dc) {
-              const uint32_t qa = q_addr + dc * q_sub_bytes + blk * (128 * 128);
-              const uint32_t ka = k_addr + dc * kKSubBytes;
+              const uint64_t dq0 = smem_desc_sw128(q_addr + dc * q_sub_bytes + blk * (128 * 128));
+              const uint64_t dk0 = smem_desc_sw128(k_addr + dc * kKSubBytes);
 #pragma unroll
               for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t dq = smem_desc_sw128(qa + kk * 32);
-                const uint64_t dk = smem_desc_sw128(ka + kk * 32);
+                const uint64_t dq = dq0 + (uint64_t)(kk * 2);         // +32 bytes in the 16-byte-unit address field
+                const uint64_t dk = dk0 + (uint64_t)(kk * 2);
                 umma_bf16(d_tmem, pass1 ? dq : dk, pass1 ? dk : dq, idesc, (dc | kk) != 0 ? 1u : 0u);
               }
             }
             umma_commit(bar_afull(as));
-            if (++as == kAccStages) { as = 0; aph ^= 1u; }
+            if (odd) { if (++ring1 == 2) { ring1 = 0; rph1 ^= 1u; } }
+            else     { if (++ring0 == 2) { ring0 = 0; rph0 ^= 1u; } }
           }
           if (ok) umma_commit(bar_kempty(ks));
           if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
         }
         if (ok) umma_commit(bar_qempty(qb));
       }
-      ++n_item;
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
+    // Two warpgroups of four warps; each owns whole key tiles (those whose running count has its parity), so a
+    // thread sees all 128 accumulator columns of its TMEM lane and no per-tile exchange between warps is needed.
     const int etid = tid - 64;
-    const int half = (warp - 2) >> 2;                  // which 64 accumulator columns this warp drains
+    const int wg = (warp - 2) >> 2;
     const int lane_grp = warp & 3;                     // TMEM lane quarter this warp may access
     const int row_in_tile = lane_grp * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
-    int as = 0;
-    uint32_t aph = 0;
+    int ring = 0;                                      // this warpgroup's ring of two accumulator stages
+    uint32_t aph = 0, tile_count = 0;
     bool ok = true;
+    auto next_stage = [&]() {
+      if (++ring == 2) { ring = 0; aph ^= 1u; }
+    };
     for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every warp meets the named barriers
-      const ScoreItem it = decode_position(p, pos, C, lane);
+      const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
       if (it.pass == 0) continue;
-      const int c0 = p.cu[it.b];
-      const int N = p.cu[it.b + 1] - c0;
+      const int N = it.N;
       const int Weff = min(p.W, N);
       const int first_win = N - Weff;                  // position of window row 0; keys <= it are visible to all rows
-      const size_t part_base = (size_t)it.unit * p.max_items * p.Ralloc;
 
       if (it.pass == 1) {
         const int nblk = (p.R + 127) / 128;
-        float* sm_m = sm_f;                            // [2][Ralloc]
-        float* sm_l = sm_f + 2 * p.Ralloc;
+        float* sm_m = sm_stat;                         // [2][Ralloc], one copy per warpgroup
+        float* sm_l = sm_stat + 2 * p.Ralloc;
         for (int r = etid; r < 2 * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
         epi_bar_sync();
-        for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
+        for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
+          if (((tile_count++) & 1u) != (uint32_t)wg || !ok) continue;
           const int t0 = tile * kTileKeys;
           const bool all_visible = t0 + kTileKeys - 1 <= first_win;
-          for (int blk = 0; blk < nblk && ok; ++blk) {
-            ok = mbar_wait(bar_afull(as), aph, abort_flag);
-            if (!ok) break;
+          for (int blk = 0; blk < nblk; ++blk) {
+            const int as = wg * 2 + ring;
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            if (!ok) continue;
             tc_fence_after();
             const int r = blk * 128 + row_in_tile;
             const bool row_ok = r < p.R && (r / p.G) < Weff;
             const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
-            float m = sm_m[half * p.Ralloc + r], lsum = sm_l[half * p.Ralloc + r];
-#pragma unroll 1
-            for (int j = 0; j < 2; ++j) {
-              const int col0 = half * 64 + j * 32;
-              float v[32];
-              tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
+            float m = sm_m[wg * p.Ralloc + r], lsum = sm_l[wg * p.Ralloc + r];
+            const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
+            uint32_t ra[32], rb[32];
+            tmem_ld32_issue(ra, t_blk);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t (&cur)[32] = (j & 1) ? rb : ra;
+              uint32_t (&nxt)[32] = (j & 1) ? ra : rb;
+              tmem_wait_ld(cur);
+              if (j + 1 < 4) tmem_ld32_issue(nxt, t_blk + (uint32_t)((j + 1) * 32));
+              const int col0 = j * 32;
               if (all_visible && row_ok) {
-                float mx = v[0];
+                float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
+                float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
 #pragma unroll
-                for (int c = 1; c < 32; ++c) mx = fmaxf(mx, v[c]);
-                const float mn = fmaxf(m, mx * p.scale_log2);
-                float s = 0.f;
+                for (int c = 4; c < 32; c += 4) {
+                  mx0 = fmaxf(mx0, __uint_as_float(cur[c]));     mx1 = fmaxf(mx1, __uint_as_float(cur[c + 1]));
+                  mx2 = fmaxf(mx2, __uint_as_float(cur[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(cur[c + 3]));
+                }
+                const float mn = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) s += exp2f(fmaf(v[c], p.scale_log2, -mn));
-                lsum = lsum * exp2f(m - mn) + s;
+                for (int c = 0; c < 32; c += 4) {
+                  s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn));
+                  s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -mn));
+                  s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -mn));
+                  s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -mn));
+                }
+                lsum = lsum * exp2f(m - mn) + ((s0 + s1) + (s2 + s3));
                 m = mn;
               } else if (col0 <= cmax) {
                 float mx = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, v[c]) : mx;
+                for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, __uint_as_float(cur[c])) : mx;
                 const float mn = fmaxf(m, mx * p.scale_log2);
                 float s = 0.f;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) s += (col0 + c <= cmax) ? exp2f(fmaf(v[c], p.scale_log2, -mn)) : 0.f;
+                for (int c = 0; c < 32; ++c)
+                  s += (col0 + c <= cmax) ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn)) : 0.f;
                 lsum = lsum * exp2f(m - mn) + s;
                 m = mn;
               }
             }
-            sm_m[half * p.Ralloc + r] = m;
-            sm_l[half * p.Ralloc + r] = lsum;
+            sm_m[wg * p.Ralloc + r] = m;
+            sm_l[wg * p.Ralloc + r] = lsum;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_aempty(as));
-            if (++as == kAccStages) { as = 0; aph ^= 1u; }
+            next_stage();
           }
         }
         epi_bar_sync();
-        const size_t slot = part_base + (size_t)it.item_in_unit * p.Ralloc;
+        const size_t slot = ((size_t)it.unit * p.max_items + it.item_in_unit) * p.Ralloc;
         for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
           const float m0 = sm_m[r], m1 = sm_m[p.Ralloc + r];
           const float M = fmaxf(m0, m1);
@@ -482,18 +495,18 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           p.part_m[slot + r] = M;
           p.part_l[slot + r] = sm_l[r] * exp2f(m0 - Mu) + sm_l[p.Ralloc + r] * exp2f(m1 - Mu);
         }
-        __threadfence();                               // this thread's statistics are visible GPU-wide ...
-        epi_bar_sync();
-        if (etid == 0 && ok && !*abort_flag) atomicAdd(p.p1_done + it.unit, 1);   // ... before the item is counted as done
+        epi_bar_sync();                                // every thread's statistics are written (CTA-wide order) ...
+        if (etid == 0 && ok && !*abort_flag) {
+          __threadfence();                             // ... made visible GPU-wide by one cumulative fence ...
+          atomicAdd(p.p1_done + it.unit, 1);           // ... before the item is counted as done
+        }
       } else {
         const int nblk = (p.Rpad + 127) / 128;
-        float* lse2 = sm_f;                            // [Ralloc]
-        float* sm_part = sm_f + p.Ralloc;              // [2][128]
+        float* lse2 = lse_buf;                         // [Ralloc] row log-sum-exps (log2 domain) of (unit, b)
         // Wait (bounded) until every pass-1 item of this unit has published its row statistics.
         if (etid == 0 && ok) {
           uint64_t t0 = 0;
-          for (uint32_t spin = 0;; ++spin) {
-            if (ld_acquire_gpu(p.p1_done + it.unit) >= C) break;
+          for (uint32_t spin = 0; ld_acquire_gpu(p.p1_done + it.unit) < C; ++spin) {
             if (*abort_flag) break;
             if ((spin & 63u) == 63u) {
               const uint64_t now = global_timer_ns();
@@ -505,67 +518,74 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         }
         epi_bar_sync();
         if (*abort_flag) ok = false;
-        for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
-          float val = INFINITY;                        // rows outside the window: exp2(x - inf) = 0
-          if (ok && r < p.R && (r / p.G) < Weff) {
-            float M = -INFINITY;
-            for (int c = 0; c < it.nch_b; ++c) M = fmaxf(M, __ldcg(p.part_m + part_base + (size_t)(it.first_item_b + c) * p.Ralloc + r));
-            float L = 0.f;
-            for (int c = 0; c < it.nch_b; ++c) {
-              const size_t o = part_base + (size_t)(it.first_item_b + c) * p.Ralloc + r;
-              L += __ldcg(p.part_l + o) * exp2f(__ldcg(p.part_m + o) - M);
+        {
+          const size_t part_base = ((size_t)it.unit * p.max_items + it.first_item_b) * p.Ralloc;
+          for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
+            float val = INFINITY;                      // rows outside the window: exp2(x - inf) = 0
+            if (ok && r < p.R && (r / p.G) < Weff) {
+              float M = -INFINITY;
+              for (int c = 0; c < it.nch_b; ++c) M = fmaxf(M, __ldcg(p.part_m + part_base + (size_t)c * p.Ralloc + r));
+              float L = 0.f;
+              for (int c = 0; c < it.nch_b; ++c) {
+                const size_t o = part_base + (size_t)c * p.Ralloc + r;
+                L += __ldcg(p.part_l + o) * exp2f(__ldcg(p.part_m + o) - M);
+              }
+              val = M + log2f(L);
             }
-            val = M + log2f(L);
+            lse2[r] = val;
           }
-          lse2[r] = val;
         }
         epi_bar_sync();
         for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
+          if (((tile_count++) & 1u) != (uint32_t)wg || !ok) continue;
           const int t = tile * kTileKeys + row_in_tile;  // this thread's key
           const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
           const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
-          float acc = 0.f;
-          for (int blk = 0; blk < nblk && ok; ++blk) {
-            ok = mbar_wait(bar_afull(as), aph, abort_flag);
-            if (!ok) break;
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          for (int blk = 0; blk < nblk; ++blk) {
+            const int as = wg * 2 + ring;
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            if (!ok) continue;
             tc_fence_after();
             const int ncols = min(128, p.Rpad - blk * 128);
-#pragma unroll 1
-            for (int j = 0; j < 2; ++j) {
-              const int col0 = half * 64 + j * 32;
-              if (col0 >= ncols) break;
-              float v[32];
-              tmem_ld32(v, t_lane + (uint32_t)(as * 128 + col0));
-              const float* ls = lse2 + blk * 128 + col0;
-              if (all_visible && col0 + 32 <= ncols) {
+            const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
+            uint32_t ra[32], rb[32];
+            tmem_ld32_issue(ra, t_blk);
 #pragma unroll
-                for (int c = 0; c < 32; c += 4) {
-                  const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                  acc += exp2f(fmaf(v[c], p.scale_log2, -l4.x));
-                  acc += exp2f(fmaf(v[c + 1], p.scale_log2, -l4.y));
-                  acc += exp2f(fmaf(v[c + 2], p.scale_log2, -l4.z));
-                  acc += exp2f(fmaf(v[c + 3], p.scale_log2, -l4.w));
-                }
-              } else {
+            for (int j = 0; j < 4; ++j) {
+              uint32_t (&cur)[32] = (j & 1) ? rb : ra;
+              uint32_t (&nxt)[32] = (j & 1) ? ra : rb;
+              const int col0 = j * 32;
+              if (col0 < ncols) {
+                tmem_wait_ld(cur);
+                if (j + 1 < 4 && col0 + 32 < ncols) tmem_ld32_issue(nxt, t_blk + (uint32_t)(col0 + 32));
+                const float* ls = lse2 + blk * 128 + col0;
+                if (all_visible && col0 + 32 <= ncols) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                  const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
-                  acc += vis ? exp2f(fmaf(v[c], p.scale_log2, -ls[c])) : 0.f;
+                  for (int c = 0; c < 32; c += 4) {
+                    const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                    a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
+                    a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
+                    a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
+                    a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
+                  }
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 32; ++c) {
+                    const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
+                    a0 += vis ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -ls[c])) : 0.f;
+                  }
                 }
               }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_aempty(as));
-            if (++as == kAccStages) { as = 0; aph ^= 1u; }
+            next_stage();
           }
-          float* part = sm_part + (tile & 1) * 128;
-          if (half == 1) part[row_in_tile] = acc;
-          epi_bar_sync();
-          if (half == 0 && ok && t < N)
-            p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + c0 + t] = acc + part[row_in_tile];
+          if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = (a0 + a1) + (a2 + a3);
         }
-        epi_bar_sync();                                // lse2 / part are reused by the next item
+        epi_bar_sync();                                // lse2 is rewritten by the next pass-2 item
       }
     }
   }
@@ -611,7 +631,7 @@ ScorePlan plan_score(const sg_shape* s) {
   pl.Ralloc = (pl.R + 127) & ~127;
   const int q_bytes = pl.Ralloc * D * 2;
   const int k_stage = kTileKeys * D * 2;
-  const int tail = 176 + 4 * pl.Ralloc * 4 + 2 * 128 * 4;
+  const int tail = (240 + 5 * pl.Ralloc * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
   const int avail = kSmemLimit - 1024 - tail;
   // Two Q buffers let the next item's queries load while the current item computes; fall back to one
   // when that would leave fewer than three K stages.
@@ -619,13 +639,16 @@ ScorePlan plan_score(const sg_shape* s) {
   pl.k_stages = (avail - 2 * q_bytes) / k_stage;
   if (pl.k_stages < 3) { pl.q_bufs = 1; pl.k_stages = (avail - q_bytes) / k_stage; }
   if (pl.k_stages > kMaxKStages) pl.k_stages = kMaxKStages;
-  pl.ok = pl.k_stages >= 2 && s->window <= 256 && pl.R <= 1024;
+  pl.ok = pl.k_stages >= 2 && s->window <= 256 && pl.R <= 1024 && s->batch <= kMaxBatchSmem;
   pl.smem_bytes = 1024 + pl.q_bufs * q_bytes + pl.k_stages * k_stage + tail;
   if (pl.smem_bytes < 120 * 1024) pl.smem_bytes = 120 * 1024;     // one CTA per SM: each CTA takes the whole TMEM
   pl.U = s->num_layers * s->num_kv_heads;
-  // chunking of the key axis: 8 tiles per item, halved while that leaves fewer than ~6 items per SM and pass
+  // Chunking of the key axis.  Above the roofline ridge (R = G*W flop per K byte vs ~218) the second read of K
+  // need not come from L2, so items are long (32 tiles) to amortise the per-item work; below it they are short
+  // (8 tiles) so that a unit's keys are still L2-resident when its pass 2 starts.  Either is halved while that
+  // leaves fewer than ~6 items per SM and pass.
   const int64_t tiles_per_unit = (int64_t)s->total_tokens / kTileKeys + s->batch;
-  int tpc = 8;
+  int tpc = pl.R >= 256 ? 32 : 8;
   while (tpc > 4 && (tiles_per_unit / tpc + s->batch) * pl.U < 6 * kNumSMs) tpc /= 2;
   pl.tiles_per_chunk = tpc;
   pl.max_items = (int)(tiles_per_unit / tpc + s->batch + 1);
