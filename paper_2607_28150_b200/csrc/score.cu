@@ -110,12 +110,25 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+// D[tmem] (+)= A[smem] * B[smem], bf16 x bf16 -> fp32, issued by one thread.  The operands are shared-memory
+// matrix descriptors given as their low words (address field); the high word is the same for every operand.
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+  if (kAccumulate) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.eq.u32 p, %1, %1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "setp.ne.u32 p, %1, %1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
+  }
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -146,16 +159,12 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
-// 128-byte swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B): 8-row groups are 1024 bytes
-// apart (stride byte offset), the leading byte offset is unused for this layout.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
-  d |= (uint64_t)(1024u >> 4) << 32;              // stride byte offset, bits [32,46)
-  d |= (uint64_t)1 << 46;                         // descriptor version for sm_100
-  d |= (uint64_t)2 << 61;                         // layout type: SWIZZLE_128B
-  return d;
-}
+// 128-byte swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).  High word: 8-row groups are 1024
+// bytes apart (stride byte offset, bits [32,46)), descriptor version 1 for sm_100 (bit 46), layout type
+// SWIZZLE_128B = 2 (bits [61,64)); the leading byte offset is unused for this layout.  Low word: the start
+// address in 16-byte units (bits [0,14)); advancing 16 elements along K inside the 128-byte span adds 2.
+constexpr uint32_t kSmemDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return (addr & 0x3FFFFu) >> 4; }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
 __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
@@ -374,16 +383,16 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const int ncols = pass1 ? 128 : min(128, p.Rpad - blk * 128);
             const uint32_t idesc = make_idesc(128, ncols);
             const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
+            const uint32_t q_lo = smem_desc_lo(q_addr + blk * (128 * 128));
+            const uint32_t k_lo = smem_desc_lo(k_addr);
+            const uint32_t a_lo = pass1 ? q_lo : k_lo, b_lo = pass1 ? k_lo : q_lo;
+            const uint32_t a_sub = (uint32_t)(pass1 ? q_sub_bytes : kKSubBytes) >> 4;
+            const uint32_t b_sub = (uint32_t)(pass1 ? kKSubBytes : q_sub_bytes) >> 4;
+            umma_bf16<false>(d_tmem, a_lo, b_lo, kSmemDescHi, idesc);
 #pragma unroll
-            for (int dc = 0; dc < kSub; ++dc) {
-              const uint64_t dq0 = smem_desc_sw128(q_addr + dc * q_sub_bytes + blk * (128 * 128));
-              const uint64_t dk0 = smem_desc_sw128(k_addr + dc * kKSubBytes);
-#pragma unroll
-              for (int kk = 0; kk < 4; ++kk) {
-                const uint64_t dq = dq0 + (uint64_t)(kk * 2);         // +32 bytes in the 16-byte-unit address field
-                const uint64_t dk = dk0 + (uint64_t)(kk * 2);
-                umma_bf16(d_tmem, pass1 ? dq : dk, pass1 ? dk : dq, idesc, (dc | kk) != 0 ? 1u : 0u);
-              }
+            for (int i = 1; i < 4 * kSub; ++i) {
+              const uint32_t dc = (uint32_t)(i >> 2), kk = (uint32_t)(i & 3);
+              umma_bf16<true>(d_tmem, a_lo + dc * a_sub + kk * 2, b_lo + dc * b_sub + kk * 2, kSmemDescHi, idesc);
             }
             umma_commit(bar_afull(as));
             if (odd) { if (++ring1 == 2) { ring1 = 0; rph1 ^= 1u; } }
