@@ -159,6 +159,36 @@ sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void
                                 int32_t* dev_status, void* stream);
 
 /*
+ * sg_split_index -- split a KV index into its local and remote parts (Algorithm 1).
+ *
+ * Defines: Algorithm 1, "KV Index Splitting and Reordering" (Section 4.2).  The KV mask holds one int8
+ * per token, shared by all heads: 0 = padding, 1 = the token's KV entries are locally available,
+ * 2 = they reside on a remote prefill node.  For every row of the KV index (one sequence, one KV head):
+ *   (1)   mask = kv_mask[kv_index]
+ *   (4,5) if `reorder`: sort the row's mask in descending order (stable: entries keep their relative
+ *         order inside a class) and apply the same order to the index, so that remote entries are
+ *         contiguous at the start of the row
+ *   (2)   local_index  = kv_index[mask == 1]
+ *   (3)   remote_index = kv_index[mask == 2]
+ * Padding entries (mask 0) are dropped from both lists; an index outside [0, N_b) sets the SG_ERR_INDEX
+ * device bit and is treated as padding.
+ *
+ * shape        num_layers must be 1 (one call per layer's KV index).
+ * kv_index     int32 [H_kv][K_tot], row segment of sequence b at cu_k[b], sequence-local positions
+ *              (the layout sg_select_topk writes for one layer); cu_k device int32 [B+1].
+ * kv_mask      int8 [T], ragged by cu_seqlens.
+ * reordered    int32 [H_kv][K_tot] or NULL: the row after steps (4)-(5) (a copy when reorder == 0).
+ * local_index, remote_index  int32 [H_kv][K_tot]: each row segment is filled from its start; the counts
+ *              go to n_local / n_remote, int32 [B][H_kv].  Entries past the counts are left untouched.
+ * The lists feed sg_sparse_decode_attn: local_index (compacted per head) is its local-lane index list,
+ * remote_index is what the prefill side gathers with sg_pack_kv.
+ */
+sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const int32_t* cu_k, int32_t total_sel,
+                         const int8_t* kv_mask, int32_t reorder, int32_t* reordered, int32_t* local_index,
+                         int32_t* remote_index, int32_t* n_local, int32_t* n_remote, int32_t* dev_status,
+                         void* stream);
+
+/*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.
  *
  * The paper has no counterpart to this call: it computes exactly what sg_score computes.  It exists

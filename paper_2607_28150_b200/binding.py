@@ -21,7 +21,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_score_static", "sg_strerror", "sg_last_cuda_error")
+            "sg_score_static", "sg_split_index", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -63,6 +63,8 @@ _lib.sg_select_topk.restype = ctypes.c_int
 _lib.sg_select_topk.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _sz, _vp, _vp]
 _lib.sg_pack_kv.restype = ctypes.c_int
 _lib.sg_pack_kv.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
+_lib.sg_split_index.restype = ctypes.c_int
+_lib.sg_split_index.argtypes = [_sp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn.restype = ctypes.c_int
 _lib.sg_sparse_decode_attn.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp,
                                        _sz, _vp, _vp]
@@ -202,3 +204,20 @@ def sg_sparse_decode_attn(shape: Shape, q: torch.Tensor, packed_k: Optional[torc
                                     _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_sparse_decode_attn")
+
+
+def sg_split_index(shape: Shape, kv_index: torch.Tensor, cu_k: torch.Tensor, total_sel: int, kv_mask: torch.Tensor,
+                   reorder: bool, reordered: Optional[torch.Tensor], local_index: torch.Tensor,
+                   remote_index: torch.Tensor, n_local: torch.Tensor, n_remote: torch.Tensor,
+                   dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Algorithm 1: split each KV index row into local (mask 1) and remote (mask 2) lists, optionally reordering
+    the row so that remote entries come first."""
+    _check(kv_index, torch.int32, "kv_index"); _check(cu_k, torch.int32, "cu_k"); _check(kv_mask, torch.int8, "kv_mask")
+    _check(reordered, torch.int32, "reordered", True); _check(local_index, torch.int32, "local_index")
+    _check(remote_index, torch.int32, "remote_index"); _check(n_local, torch.int32, "n_local")
+    _check(n_remote, torch.int32, "n_remote"); _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_split_index(ctypes.byref(shape), _ptr(kv_index), cu_k.data_ptr(), total_sel, _ptr(kv_mask),
+                             1 if reorder else 0, _ptr(reordered), _ptr(local_index), _ptr(remote_index),
+                             n_local.data_ptr(), n_remote.data_ptr(), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_split_index")
