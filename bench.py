@@ -388,7 +388,7 @@ def run_ours(args):
     cpu = None
     if not args.no_cpu_baseline:
         import oracle
-        layers = list(range(min(4, L)))
+        layers = list(range(min(16, L)))            # about 10-30 s of CPU work on the 8B-shaped workload
         t = oracle_sample(cfg, layers)
         fr = len(layers) / L
         cpu = {"value": sp_bytes * fr / (t["select"] + t["pack"]) / 1e9, "unit": UNIT, "cores": oracle.max_threads(),

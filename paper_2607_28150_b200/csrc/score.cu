@@ -14,7 +14,7 @@
 //
 // One persistent kernel runs both passes: warp 0 feeds Q and 128-key K tiles with TMA into
 // 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM accumulator
-// stages (a ring of two per epilogue warpgroup), warps 2-9 (two warpgroups, each owning alternate key tiles) drain them with pipelined
+// stages (one per epilogue warpgroup), the epilogue warps (four warpgroups, each owning every fourth key tile) drain them with pipelined
 // tcgen05.ld.  The score matrix never leaves the SM.  Work items (a pass, a layer/KV head, a chunk of
 // key tiles of one sequence) are laid out so that pass 2 of a (layer, KV head) unit follows its pass 1
 // by a lag of a few units: close enough that the unit's keys are still in L2 for the second read
@@ -33,9 +33,11 @@
 namespace sg {
 namespace {
 
-constexpr int kScoreThreads = 320;        // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-9: epilogue
-constexpr int kEpiThreads = 256;
+constexpr int kEpiGroups = 4;             // epilogue warpgroups (four warps each, one per TMEM lane quarter)
+constexpr int kEpiThreads = 128 * kEpiGroups;
+constexpr int kScoreThreads = 64 + kEpiThreads;   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
 constexpr int kTileKeys = 128;
+constexpr int kRing = 4 / kEpiGroups;        // accumulator stages per epilogue warpgroup
 constexpr int kAccStages = 4;             // 4 x 128 fp32 columns = the whole 512-column TMEM
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxKStages = 4;
@@ -237,8 +239,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 28 * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 28 * 8 + 4);
   float* lse_buf = reinterpret_cast<float*>(tail + 240);              // [Ralloc] row log-sum-exps of the current pass-2 item
-  float* sm_stat = lse_buf + p.Ralloc;                            // pass 1: m[2][Ralloc], l[2][Ralloc]
-  int* s_cu = reinterpret_cast<int*>(sm_stat + 4 * p.Ralloc);         // [B+1]
+  float* sm_stat = lse_buf + p.Ralloc;                            // pass 1: m[groups][Ralloc], l[groups][Ralloc]
+  float* sm_part = sm_stat + 2 * kEpiGroups * p.Ralloc;               // pass 2, several blocks per tile: [2][groups][128] partial column sums
+  int* s_cu = reinterpret_cast<int*>(sm_part + 2 * kEpiGroups * 128);         // [B+1]
   int* s_prefix = s_cu + p.B + 1;                                     // [B+1]
 
   auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
@@ -354,8 +357,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     // only, so no waiter ever falls more than one mbarrier phase behind.
     if (lane == 0) {
       int ks = 0, n_item = 0;
-      int ring0 = 0, ring1 = 0;
-      uint32_t kph = 0, rph0 = 0, rph1 = 0, tile_count = 0;
+      uint32_t kph = 0, ringbits = 0, phbits = 0, tile_count = 0;   // one ring-index bit and one phase bit per warpgroup
       bool ok = true;
       for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
         const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
@@ -374,10 +376,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           if (!ok) break;
           tc_fence_after();
           const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
-          const bool odd = ((tile_count++) & 1u) != 0;
+          const bool blockwise = nblk > 1;                 // several blocks per key tile: deal blocks, not tiles
+          uint32_t wgsel = blockwise ? 0u : (tile_count++) % kEpiGroups;
           for (int blk = 0; blk < nblk && ok; ++blk) {
-            const int as = odd ? 2 + ring1 : ring0;
-            ok = mbar_wait(bar_aempty(as), (odd ? rph1 : rph0) ^ 1u, abort_flag);
+            if (blockwise) wgsel = (tile_count++) % kEpiGroups;
+            const uint32_t ridx = kRing == 2 ? ((ringbits >> wgsel) & 1u) : 0u;
+            const int as = (int)(wgsel * kRing + ridx);
+            ok = mbar_wait(bar_aempty(as), ((phbits >> wgsel) & 1u) ^ 1u, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const int ncols = pass1 ? 128 : min(128, p.Rpad - blk * 128);
@@ -395,8 +400,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               umma_bf16<true>(d_tmem, a_lo + dc * a_sub + kk * 2, b_lo + dc * b_sub + kk * 2, kSmemDescHi, idesc);
             }
             umma_commit(bar_afull(as));
-            if (odd) { if (++ring1 == 2) { ring1 = 0; rph1 ^= 1u; } }
-            else     { if (++ring0 == 2) { ring0 = 0; rph0 ^= 1u; } }
+            if (kRing == 2) { ringbits ^= 1u << wgsel; if (ridx == 1u) phbits ^= 1u << wgsel; }
+            else phbits ^= 1u << wgsel;
           }
           if (ok) umma_commit(bar_kempty(ks));
           if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
@@ -406,7 +411,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    // Two warpgroups of four warps; each owns whole key tiles (those whose running count has its parity), so a
+    // Warpgroups of four warps; each owns whole key tiles (every kEpiGroups-th of the CTA's running count), so a
     // thread sees all 128 accumulator columns of its TMEM lane and no per-tile exchange between warps is needed.
     const int etid = tid - 64;
     const int wg = (warp - 2) >> 2;
@@ -417,7 +422,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     uint32_t aph = 0, tile_count = 0;
     bool ok = true;
     auto next_stage = [&]() {
-      if (++ring == 2) { ring = 0; aph ^= 1u; }
+      if (++ring == kRing) { ring = 0; aph ^= 1u; }
     };
     for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every warp meets the named barriers
       const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
@@ -428,16 +433,18 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
 
       if (it.pass == 1) {
         const int nblk = (p.R + 127) / 128;
-        float* sm_m = sm_stat;                         // [2][Ralloc], one copy per warpgroup
-        float* sm_l = sm_stat + 2 * p.Ralloc;
-        for (int r = etid; r < 2 * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
+        float* sm_m = sm_stat;                         // [groups][Ralloc], one copy per warpgroup
+        float* sm_l = sm_stat + kEpiGroups * p.Ralloc;
+        for (int r = etid; r < kEpiGroups * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
         epi_bar_sync();
         for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
-          if (((tile_count++) & 1u) != (uint32_t)wg || !ok) continue;
+          const bool blockwise = nblk > 1;
+          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t0 = tile * kTileKeys;
           const bool all_visible = t0 + kTileKeys - 1 <= first_win;
           for (int blk = 0; blk < nblk; ++blk) {
-            const int as = wg * 2 + ring;
+            if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+            const int as = wg * kRing + ring;
             if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
             if (!ok) continue;
             tc_fence_after();
@@ -446,15 +453,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
             float m = sm_m[wg * p.Ralloc + r], lsum = sm_l[wg * p.Ralloc + r];
             const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
-            uint32_t ra[32], rb[32];
-            tmem_ld32_issue(ra, t_blk);
-#pragma unroll
+            uint32_t cur[32];                            // (four warps per scheduler hide the TMEM load latency)
+#pragma unroll 1
             for (int j = 0; j < 4; ++j) {
-              uint32_t (&cur)[32] = (j & 1) ? rb : ra;
-              uint32_t (&nxt)[32] = (j & 1) ? ra : rb;
-              tmem_wait_ld(cur);
-              if (j + 1 < 4) tmem_ld32_issue(nxt, t_blk + (uint32_t)((j + 1) * 32));
               const int col0 = j * 32;
+              tmem_ld32_issue(cur, t_blk + (uint32_t)col0);
+              tmem_wait_ld(cur);
               if (all_visible && row_ok) {
                 float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
                 float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
@@ -498,11 +502,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         epi_bar_sync();
         const size_t slot = ((size_t)it.unit * p.max_items + it.item_in_unit) * p.Ralloc;
         for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
-          const float m0 = sm_m[r], m1 = sm_m[p.Ralloc + r];
-          const float M = fmaxf(m0, m1);
+          float M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < kEpiGroups; ++w) M = fmaxf(M, sm_m[w * p.Ralloc + r]);
           const float Mu = M == -INFINITY ? 0.f : M;
+          float L = 0.f;
+#pragma unroll
+          for (int w = 0; w < kEpiGroups; ++w) L += sm_l[w * p.Ralloc + r] * exp2f(sm_m[w * p.Ralloc + r] - Mu);
           p.part_m[slot + r] = M;
-          p.part_l[slot + r] = sm_l[r] * exp2f(m0 - Mu) + sm_l[p.Ralloc + r] * exp2f(m1 - Mu);
+          p.part_l[slot + r] = L;
         }
         epi_bar_sync();                                // every thread's statistics are written (CTA-wide order) ...
         if (etid == 0 && ok && !*abort_flag) {
@@ -546,28 +554,27 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         }
         epi_bar_sync();
         for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
-          if (((tile_count++) & 1u) != (uint32_t)wg || !ok) continue;
+          const bool blockwise = nblk > 1;
+          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t = tile * kTileKeys + row_in_tile;  // this thread's key
           const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
           const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
           float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
           for (int blk = 0; blk < nblk; ++blk) {
-            const int as = wg * 2 + ring;
+            if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+            const int as = wg * kRing + ring;
             if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
             if (!ok) continue;
             tc_fence_after();
             const int ncols = min(128, p.Rpad - blk * 128);
             const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
-            uint32_t ra[32], rb[32];
-            tmem_ld32_issue(ra, t_blk);
-#pragma unroll
+            uint32_t cur[32];
+#pragma unroll 1
             for (int j = 0; j < 4; ++j) {
-              uint32_t (&cur)[32] = (j & 1) ? rb : ra;
-              uint32_t (&nxt)[32] = (j & 1) ? ra : rb;
               const int col0 = j * 32;
               if (col0 < ncols) {
+                tmem_ld32_issue(cur, t_blk + (uint32_t)col0);
                 tmem_wait_ld(cur);
-                if (j + 1 < 4 && col0 + 32 < ncols) tmem_ld32_issue(nxt, t_blk + (uint32_t)(col0 + 32));
                 const float* ls = lse2 + blk * 128 + col0;
                 if (all_visible && col0 + 32 <= ncols) {
 #pragma unroll
@@ -592,7 +599,18 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             if (lane == 0) mbar_arrive(bar_aempty(as));
             next_stage();
           }
-          if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = (a0 + a1) + (a2 + a3);
+          float total = (a0 + a1) + (a2 + a3);
+          if (blockwise) {
+            // the tile's column blocks were dealt to different warpgroups: add their partial column sums
+            float* part = sm_part + (tile & 1) * (kEpiGroups * 128);
+            part[wg * 128 + row_in_tile] = total;
+            epi_bar_sync();
+            if (wg != 0) continue;
+            total = 0.f;
+#pragma unroll
+            for (int w = 0; w < kEpiGroups; ++w) total += part[w * 128 + row_in_tile];
+          }
+          if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
         }
         epi_bar_sync();                                // lse2 is rewritten by the next pass-2 item
       }
@@ -640,7 +658,7 @@ ScorePlan plan_score(const sg_shape* s) {
   pl.Ralloc = (pl.R + 127) & ~127;
   const int q_bytes = pl.Ralloc * D * 2;
   const int k_stage = kTileKeys * D * 2;
-  const int tail = (240 + 5 * pl.Ralloc * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
+  const int tail = (240 + (1 + 2 * kEpiGroups) * pl.Ralloc * 4 + 2 * kEpiGroups * 128 * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
   const int avail = kSmemLimit - 1024 - tail;
   // Two Q buffers let the next item's queries load while the current item computes; fall back to one
   // when that would leave fewer than three K stages.
