@@ -161,6 +161,147 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelPa
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Register-resident variant for rows of up to 32768 tokens: thread t owns E consecutive positions
+// [t*E, (t+1)*E) and keeps their keys in registers (the row is read coalesced into a padded shared-memory
+// staging buffer first, then each thread picks up its segment with 16-byte loads).  Three MSB-first
+// passes (11 + 11 + 10 bits) find the k-th largest key; after the first pass only the few keys inside
+// the threshold bin take part.  Because ownership is contiguous, one block-wide prefix sum over
+// per-thread (greater, equal) counts gives every thread the output offset of its first selected
+// position, and it writes its positions in ascending order.
+constexpr int kRegBins = 2048;
+constexpr int kRegCopies = 2;
+
+// Block-wide exclusive prefix sum of one value per thread (T threads); `wsum` holds 2*T/32 words.
+template <int T>
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* wsum, int lane, int warp) {
+  uint32_t inc = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t u = __shfl_up_sync(0xffffffffu, inc, off);
+    if (lane >= off) inc += u;
+  }
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t w = lane < T / 32 ? wsum[lane] : 0u;
+    uint32_t wi = w;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t u = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += u;
+    }
+    if (lane < T / 32) wsum[T / 32 + lane] = wi - w;
+  }
+  __syncthreads();
+  return wsum[T / 32 + warp] + inc - v;
+}
+
+template <int E, int T>
+__global__ void __launch_bounds__(T) select_topk_reg_kernel(const SelParams p) {
+  extern __shared__ __align__(16) uint32_t smem[];
+  uint32_t* hist = smem;                               // [kRegCopies][kRegBins]
+  uint32_t* wsum = hist + kRegCopies * kRegBins;       // [2][T/32]
+  uint32_t* sh = wsum + 2 * (T / 32);                  // [0] chosen bin, [1] remaining need  (8 words)
+  uint32_t* stage = sh + 8;                            // [T][E + 4] keys, each thread's segment padded by 16 bytes
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = blockIdx.x;
+  const int l = row / (p.B * p.Hkv);
+  const int rem = row - l * (p.B * p.Hkv);
+  const int b = rem / p.Hkv;
+  const int g = rem - b * p.Hkv;
+  const int c0 = p.cu[b];
+  const int N = p.cu[b + 1] - c0;
+  const int ck = p.cu_k[b];
+  const int kb = p.cu_k[b + 1] - ck;
+  if (kb <= 0) return;
+  int32_t* out = p.sel_idx + ((int64_t)l * p.Hkv + g) * p.K_tot + ck;
+  if (kb >= N) {                                      // whole prompt (or an over-sized budget)
+    if (kb > N && tid == 0) raise(p.dev_status, SG_ERR_INVALID);
+    for (int j = tid; j < kb; j += T) out[j] = j < N ? j : -1;
+    return;
+  }
+  const uint32_t* x = reinterpret_cast<const uint32_t*>(p.importance) + ((int64_t)l * p.Hkv + g) * p.T + c0;
+  for (int i = tid; i < kRegCopies * kRegBins; i += T) hist[i] = 0;
+  {
+    uint32_t v[E];                                     // all E loads of the thread are issued before the first store
+#pragma unroll
+    for (int e = 0; e < E; ++e) { const int i = tid + e * T; v[e] = i < N ? __ldg(x + i) : 0u; }
+#pragma unroll
+    for (int e = 0; e < E; ++e) { const int i = tid + e * T; stage[i + 4 * (i / E)] = i < N ? order_key(v[e]) : 0u; }
+  }
+  __syncthreads();
+  const int first = tid * E;
+  uint32_t key[E];
+#pragma unroll
+  for (int e = 0; e < E; e += 4) {
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + tid * (E + 4) + e);
+    key[e] = v.x; key[e + 1] = v.y; key[e + 2] = v.z; key[e + 3] = v.w;
+  }
+
+  uint32_t prefix = 0, decided = 0, need = (uint32_t)kb;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const int nbins = pass == 2 ? 1024 : 2048;
+    const int copies = pass == 0 ? kRegCopies : 1;     // later passes see few candidates: one copy is enough
+    uint32_t* my_hist = hist + (warp % copies) * kRegBins;
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+      if (first + e < N && (key[e] & decided) == prefix) atomicAdd(&my_hist[(key[e] >> shift) & (uint32_t)(nbins - 1)], 1u);
+    __syncthreads();
+    // suffix search: thread t looks at bins nbins-1-t*bpt ... (descending); the bin holding the need-th largest
+    const int bpt = nbins / T > 0 ? nbins / T : 1;
+    uint32_t c[kRegBins / T > 0 ? kRegBins / T : 1];
+    uint32_t ssum = 0;
+#pragma unroll
+    for (int i = 0; i < (kRegBins / T > 0 ? kRegBins / T : 1); ++i) {
+      const int bin = nbins - 1 - (tid * bpt + i);
+      c[i] = 0;
+      if (i < bpt && bin >= 0) {
+        for (int k = 0; k < copies; ++k) { c[i] += hist[k * kRegBins + bin]; hist[k * kRegBins + bin] = 0; }   // read and clear for the next pass
+      }
+      ssum += c[i];
+    }
+    const uint32_t exc = block_exclusive_scan<T>(ssum, wsum, lane, warp);   // candidates in bins above this thread's
+    if (exc < need && need <= exc + ssum) {
+      uint32_t run = exc;
+#pragma unroll
+      for (int i = 0; i < (kRegBins / T > 0 ? kRegBins / T : 1); ++i) {
+        if (run < need && need <= run + c[i]) { sh[0] = (uint32_t)(nbins - 1 - (tid * bpt + i)); sh[1] = need - run; }
+        run += c[i];
+      }
+    }
+    __syncthreads();
+    prefix |= sh[0] << shift;
+    decided |= (uint32_t)(nbins - 1) << shift;
+    need = sh[1];
+  }
+  const uint32_t tau = prefix, need_eq = need;
+
+  // per-thread counts, packed (greater in the low half, equal in the high half), block-wide exclusive prefix
+  uint32_t cnt = 0;
+#pragma unroll
+  for (int e = 0; e < E; ++e)
+    if (first + e < N) cnt += (key[e] > tau ? 1u : 0u) + (key[e] == tau ? 0x10000u : 0u);
+  const uint32_t before = block_exclusive_scan<T>(cnt, wsum, lane, warp);
+  uint32_t gt_before = before & 0xffffu, eq_before = before >> 16;
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    if (first + e < N) {
+      const bool is_gt = key[e] > tau, is_eq = key[e] == tau;
+      if (is_gt || (is_eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = first + e;
+      gt_before += is_gt ? 1u : 0u;
+      eq_before += is_eq ? 1u : 0u;
+    }
+  }
+}
+
+template <int E, int T>
+constexpr int select_reg_smem_bytes() { return (kRegCopies * kRegBins + 2 * (T / 32) + 8 + T * (E + 4)) * 4; }
+
 }  // namespace
 }  // namespace sg
 
@@ -189,13 +330,27 @@ extern "C" sg_status sg_select_topk(const sg_shape* shape, const float* importan
   const int64_t rows = (int64_t)shape->num_layers * shape->batch * shape->num_kv_heads;
   if (rows > 0x7fffffffLL) return SG_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (shape->max_seqlen <= kSelKeyCap) {
+#define SG_LAUNCH_SELECT_REG(E, T)                                                         \
+  do {                                                                                   \
+    SG_ENSURE_SMEM((select_topk_reg_kernel<E, T>), (select_reg_smem_bytes<E, T>()));      \
+    select_topk_reg_kernel<E, T><<<(unsigned)rows, T, select_reg_smem_bytes<E, T>(), s>>>(p); \
+  } while (0)
+  if (shape->max_seqlen <= 4096) {
+    SG_LAUNCH_SELECT_REG(8, 512);
+  } else if (shape->max_seqlen <= 8192) {
+    SG_LAUNCH_SELECT_REG(16, 512);
+  } else if (shape->max_seqlen <= 16384) {
+    SG_LAUNCH_SELECT_REG(16, 1024);
+  } else if (shape->max_seqlen <= 32768) {
+    SG_LAUNCH_SELECT_REG(32, 1024);
+  } else if (shape->max_seqlen <= kSelKeyCap) {
     const int smem = kSelFixedSmem + shape->max_seqlen * 4;
     SG_ENSURE_SMEM(select_topk_kernel<true>, smem);
     select_topk_kernel<true><<<(unsigned)rows, kSelThreads, smem, s>>>(p);
   } else {
     select_topk_kernel<false><<<(unsigned)rows, kSelThreads, kSelFixedSmem, s>>>(p);
   }
+#undef SG_LAUNCH_SELECT_REG
   SG_CUDA_TRY(cudaGetLastError());
   return SG_OK;
 }

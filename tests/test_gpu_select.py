@@ -21,6 +21,8 @@ def check(x, lens, ks, expect_status=0):
     ((8192,), (820,), 2, 8),
     ((33, 1, 700, 5000), (5, 1, 0, 4999), 2, 3),
     ((32768,), (2048,), 1, 2),
+    ((12000, 9000), (1200, 1), 1, 2),     # 16 keys per thread in registers
+    ((40000,), (4000,), 1, 1),            # shared-memory key buffer variant
     ((60000,), (3000,), 1, 1),            # longer than the shared-memory key buffer: global-memory path
 ])
 def test_select_random_values(lens, ks, L, Hkv):
