@@ -33,7 +33,11 @@ UNIT = "GB/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes; None where no capture exists).  Keyed by workload then kernel.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/kernels_ncu_set_full.md, case A (8 of the 32 layers): per-launch bytes scaled x4 where a launch
+    # covers all layers; the decode call is per layer.  (pack: its stores were still in L2 when the capture ended.)
+    "c2": {"score": 4 * (136.617e6 + 6.328e6), "select": 4 * 2.125e6, "pack": 4 * (27.097e6 + 0.131e6), "decode": 5.163e6},
+}
 
 
 def load_peaks():
@@ -369,7 +373,7 @@ def run_ours(args):
                 "frac": a / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy)", "ms_per_step": ms,
                 "launches_per_step": launches, "traffic": ncu.get(name)}
     roofs = {
-        "score": hbm("score", work["score"]["bytes"], st["score"], 2),
+        "score": hbm("score", work["score"]["bytes"], st["score"], 1),
         "select": hbm("select", work["select"]["bytes"], st["select"], 1),
         "pack": hbm("pack", work["pack"]["bytes"], st["pack"], 1),
     }
@@ -380,7 +384,7 @@ def run_ours(args):
         roofs["score"].update(bound="tensor", achieved=roofs["score"]["tensor_tflops"], peak=tc_peak, unit="TFLOP/s",
                               frac=roofs["score"]["tensor_frac_of_sustained"], peak_source=peaks["source"] + " (sustained bf16)")
     if ncalls_dec:
-        roofs["decode"] = hbm("decode", work["decode_call"]["bytes"] * ncalls_dec, st["decode"], 2 * ncalls_dec)
+        roofs["decode"] = hbm("decode", work["decode_call"]["bytes"] * ncalls_dec, st["decode"], ncalls_dec)
         roofs["decode"]["us_per_call"] = 1e3 * st["decode"] / ncalls_dec
     dominant = max(roofs.values(), key=lambda r: r["ms_per_step"])
 
@@ -411,7 +415,7 @@ def run_ours(args):
         "stage_ms": st,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
-        "gpu_launches": args.steps * (4 + 2 * ncalls_dec),
+        "gpu_launches": args.steps * (3 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
         "dev_status": status, "setup_s": gen_s,
     }
