@@ -345,11 +345,8 @@ def run_ours(args):
     ms_e2e, st_e = timed(True, e2e_steps, 1)
     status = hp.read_status()
 
-    if world > 1:
-        gather = [None] * world
-        dist.all_gather_object(gather, {"st": st, "st_e": st_e})
-        st = {k: max(gg["st"][k] for gg in gather) for k in st}
-        st_e = {k: max(gg["st_e"][k] for gg in gather) for k in st_e}
+    from paper_2607_28150_b200 import replicas
+    st, st_e = replicas.max_over_ranks(st), replicas.max_over_ranks(st_e)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
