@@ -195,6 +195,62 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------- CUDA arm
+
+def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (128, 1.0, 0.5)), calls=16):
+    """sg_sparse_decode_attn alone on points of the decode-heavy sweep (B sequences of 4096 tokens, `sel` of the
+    prompt required, `rho` of that index-addressed): the sizes at which the kernel can reach the HBM roofline.
+    K/V are seeded N(0,1) bf16 generated on the device; the packed buffer is built by sg_pack_kv; every call of a
+    timed graph reads more than L2 holds.  Returns one dict per point."""
+    import torch
+    from paper_2607_28150_b200 import binding as sg, workloads as wl
+    from paper_2607_28150_b200.pipeline import as_device
+    out = []
+    gen = torch.Generator(device=dev)
+    for (B, sel, rho) in points:
+        cfg = wl.decode_sweep(B, sel, rho)
+        Hq, Hkv, d, N = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.seqlens[0]
+        T = B * N
+        gen.manual_seed(5000 + B)
+        k = torch.randn((T, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        v = torch.randn((T, Hkv, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        q = torch.randn((B, Hq, d), generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        sel_idx, ck, loc, cl = wl.make_index_split(cfg, 0, 0, cfg.budgets(), cfg.n_local())
+        Ktot, NL = int(ck[-1]), int(cl[-1])
+        cu = as_device(cfg.cu_seqlens(), dev)
+        d_ck, d_cl = as_device(ck, dev), as_device(cl, dev)
+        shp = sg.make_shape(1, Hq, Hkv, d, 1, cu, T, N)
+        pk = torch.empty((max(Ktot, 1) * Hkv, d), dtype=torch.bfloat16, device=dev)
+        pv = torch.empty_like(pk)
+        if Ktot:
+            sg.sg_pack_kv(shp, k, v, as_device(sel_idx, dev), d_ck, Ktot, pk, pv)
+        d_loc = as_device(loc, dev) if NL else None
+        o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=dev)
+        call = lambda: sg.sg_sparse_decode_attn(shp, q, pk if Ktot else None, pv if Ktot else None, d_ck, Ktot, k, v,
+                                                d_loc, d_cl, NL, o)
+        call()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(calls):
+                call()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = float("inf")
+        for _ in range(3):
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        us = best * 1e3 / calls
+        nbytes = Hkv * (2 * (Ktot + NL) * d * 2 + NL * 4) + 2 * B * Hq * d * 2
+        gbs = nbytes / us / 1e3
+        out.append({"batch": B, "sel": sel, "rho": rho, "n_sel": Ktot // B, "n_loc": NL // B, "us_per_call": us,
+                    "bytes_per_call": nbytes, "achieved_gbs": gbs, "frac_of_copy_peak": gbs / peaks["hbm_gbs"],
+                    "tokens_per_s": B / (us * 1e-6)})
+        del k, v, pk, pv
+        torch.cuda.empty_cache()
+    return out
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -340,9 +396,9 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     ms_step, st = timed(False, args.steps, max(3, args.warmup))
-    clocks = sampler.stop() if rank == 0 else {}
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     ms_e2e, st_e = timed(True, e2e_steps, 1)
+    clocks = sampler.stop() if rank == 0 else {}       # sampled over both timed regions
     status = hp.read_status()
 
     from paper_2607_28150_b200 import replicas
@@ -399,13 +455,20 @@ def run_ours(args):
                "decode_tokens_per_s": B * fr / t["decode"] if t["decode"] > 0 else None,
                "score_tflops": work["score"]["flops"] * fr / t["score"] / 1e12}
 
+    kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
+    sweep = None
+    if args.workload == "c2" and not args.no_decode_sweep and world == 1:
+        del d_k, d_v, h_k, h_v
+        torch.cuda.empty_cache()
+        sweep = decode_sweep_points(dev, peaks)
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": "%s: L=%d B=%d Hq=%d Hkv=%d d=%d W=%d T=%d K_tot=%d n_loc=%d decode_steps=%d" % (
                        cfg.name, L, B, Hq, Hkv, d, W, T, Ktot, NL, nsteps_dec),
-                   "l2": "inputs larger than L2 (K+V caches %.0f MiB); no flush" % ((h_k.numel() + h_v.numel()) * 2 / 2**20),
+                   "l2": "inputs larger than L2 (K+V caches %.0f MiB); no flush" % kv_mib,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "decode": "one sg_sparse_decode_attn call per layer per step, replayed from a CUDA graph"},
         "decode_tokens_per_s": dec_tok,
@@ -414,7 +477,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (3 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "dev_status": status, "setup_s": gen_s,
+        "decode_sweep": sweep, "dev_status": status, "setup_s": gen_s,
     }
     print(json.dumps(line))
     if world > 1:
@@ -436,6 +499,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode-sweep", action="store_true", help="skip the extra decode-only points (c2 only)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
