@@ -144,3 +144,38 @@ def split_index(kv_index, kv_mask, cu_seqlens, cu_k, reorder: bool = True):
     if rc:
         raise RuntimeError("sgo_split_index failed: %d" % rc)
     return reordered, loc, rem, nl, nr
+
+
+def profile_accumulate(counts, kv_index, cu_seqlens, cu_k):
+    """counts int32 [H_kv][T] += 1 at every entry of kv_index int32 [H_kv][K_tot] (in place; returns counts)."""
+    c, idx, cu, ck = _c(counts, np.int32), _c(kv_index, np.int32), _c(cu_seqlens, np.int32), _c(cu_k, np.int32)
+    assert c is counts or np.shares_memory(c, counts)
+    Hkv, T = c.shape
+    rc = _load().sgo_profile_accumulate(cu.shape[0] - 1, Hkv, _p(cu), _p(ck), _p(idx), _p(c))
+    if rc:
+        raise RuntimeError("sgo_profile_accumulate failed: %d" % rc)
+    return counts
+
+
+def block_importance(counts, cu_seqlens, num_blocks: int) -> np.ndarray:
+    """Eq. 1: float32 [L][M] from selection counts int32 [L][H_kv][T]."""
+    c, cu = _c(counts, np.int32), _c(cu_seqlens, np.int32)
+    L, Hkv, T = c.shape
+    out = np.zeros((L, num_blocks), dtype=np.float32)
+    _load().sgo_block_importance(L, cu.shape[0] - 1, Hkv, num_blocks, _p(cu), _p(c), _p(out))
+    return out
+
+
+def transfer_budget(num_layers: int, num_blocks: int, t_prefill: float, t_transfer: float) -> int:
+    """Eq. 2 with its clip to [2M, LM]."""
+    lib = _load()
+    lib.sgo_transfer_budget.restype = ctypes.c_int64
+    return int(lib.sgo_transfer_budget(num_layers, num_blocks, ctypes.c_double(t_prefill), ctypes.c_double(t_transfer)))
+
+
+def proactive_mask(cu_seqlens, num_blocks: int, layer: int, selected) -> np.ndarray:
+    """int8 [T]: 1 for tokens of layer `layer` whose block is in `selected` (flat ids l*M+m, ascending), else 2."""
+    cu, sel = _c(cu_seqlens, np.int32), _c(selected, np.int32)
+    mask = np.zeros(int(cu[-1]), dtype=np.int8)
+    _load().sgo_proactive_mask(cu.shape[0] - 1, num_blocks, _p(cu), layer, _p(sel), sel.shape[0], _p(mask))
+    return mask

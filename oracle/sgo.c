@@ -324,3 +324,78 @@ int sgo_split_index(int B, int Hkv, const int32_t *cu, const int32_t *cu_k, cons
         }
     return bad;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Profile-based proactive selection (Section 4.1).
+ *
+ * Block of a token: every layer's cache is partitioned along the sequence into M blocks; token t of
+ * a sequence of length N belongs to block floor(t * M / N), so block sizes differ by at most one.
+ */
+static int64_t block_of(int64_t t, int64_t N, int64_t M) { return t * M / N; }
+
+/* S(e): "the number of times entry e is selected in the decoding stage during the offline profiling".
+ * Adds one to counts[g][cu[b] + t] for every entry t of the KV index (one layer, one decode step).
+ * kv_index int32 [Hkv][K_tot] with prefix sums cu_k; counts int32 [Hkv][T]. */
+int sgo_profile_accumulate(int B, int Hkv, const int32_t *cu, const int32_t *cu_k, const int32_t *kv_index,
+                           int32_t *counts) {
+    const int64_t T = cu[B], K_tot = cu_k[B];
+    int bad = 0;
+    for (int g = 0; g < Hkv; ++g)
+        for (int b = 0; b < B; ++b)
+            for (int j = cu_k[b]; j < cu_k[b + 1]; ++j) {
+                const int32_t t = kv_index[(int64_t)g * K_tot + j];
+                if (t < 0 || t >= cu[b + 1] - cu[b]) { bad = 3; continue; }
+                counts[(int64_t)g * T + cu[b] + t] += 1;
+            }
+    return bad;
+}
+
+/* Eq. 1: I[l][m] = +inf for l = 0, 1; otherwise the mean of S(e) over the entries of block B_{l,m}
+ * (all tokens of the block, all KV heads, all profiled sequences).  An empty block gets 0.
+ * counts int32 [L][Hkv][T]; importance float [L][M].  The mean is a double division rounded to float. */
+int sgo_block_importance(int L, int B, int Hkv, int M, const int32_t *cu, const int32_t *counts, float *importance) {
+    const int64_t T = cu[B];
+    for (int l = 0; l < L; ++l)
+        for (int m = 0; m < M; ++m) {
+            if (l < 2) { importance[(int64_t)l * M + m] = INFINITY; continue; }
+            int64_t sum = 0, entries = 0;
+            for (int b = 0; b < B; ++b) {
+                const int64_t N = cu[b + 1] - cu[b];
+                for (int64_t t = 0; t < N; ++t) {
+                    if (block_of(t, N, M) != m) continue;
+                    entries += Hkv;
+                    for (int g = 0; g < Hkv; ++g) sum += counts[((int64_t)l * Hkv + g) * T + cu[b] + t];
+                }
+            }
+            importance[(int64_t)l * M + m] = entries ? (float)((double)sum / (double)entries) : 0.0f;
+        }
+    return 0;
+}
+
+/* Eq. 2: K_r = M (L-1) T_p / T_t, the number of blocks whose transfer overlaps the prefill of all but the first
+ * transformer block; clipped to [2M, LM] so that the first two layers always go.  Rounded down. */
+int64_t sgo_transfer_budget(int L, int M, double T_p, double T_t) {
+    double k = (double)M * (double)(L - 1) * T_p / T_t;
+    const double lo = 2.0 * M, hi = (double)L * M;
+    if (!(k >= lo)) k = lo;          /* also catches NaN */
+    if (k > hi) k = hi;
+    if (L < 2) k = hi;
+    return (int64_t)floor(k);
+}
+
+/* KV mask of one layer after the proactive transfer (Section 4.2: 1 = locally available, 2 = on the remote
+ * prefill node): tokens of the blocks of layer l that are in the global top-K_r set are local, the rest remote.
+ * selected int32 [K_r]: flat block ids l*M + m in ascending order.  mask int8 [T]. */
+int sgo_proactive_mask(int B, int M, const int32_t *cu, int layer, const int32_t *selected, int K_r, int8_t *mask) {
+    for (int b = 0; b < B; ++b) {
+        const int64_t N = cu[b + 1] - cu[b];
+        for (int64_t t = 0; t < N; ++t) {
+            const int32_t id = (int32_t)((int64_t)layer * M + block_of(t, N, M));
+            int8_t v = 2;
+            for (int j = 0; j < K_r; ++j)
+                if (selected[j] == id) { v = 1; break; }
+            mask[cu[b] + t] = v;
+        }
+    }
+    return 0;
+}

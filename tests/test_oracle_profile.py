@@ -1,0 +1,89 @@
+"""Pins for the oracle's profile-based proactive selection (Section 4.1: Eq. 1, Eq. 2, top-K_r blocks; Section 4.2 mask)."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import cu_of
+
+
+def test_accumulate_counts_each_selection_once():
+    cu, ck = cu_of((5, 3)), cu_of((2, 3))
+    idx = np.array([[0, 4, 0, 1, 2], [1, 2, 0, 1, 2]], dtype=np.int32)
+    c = np.zeros((2, 8), dtype=np.int32)
+    oracle.profile_accumulate(c, idx, cu, ck)
+    oracle.profile_accumulate(c, idx, cu, ck)
+    want = np.zeros((2, 8), dtype=np.int32)
+    want[0, [0, 4]] = 2; want[0, [5, 6, 7]] = 2
+    want[1, [1, 2]] = 2; want[1, [5, 6, 7]] = 2
+    assert np.array_equal(c, want)
+    assert c.sum() == 2 * idx.size
+
+
+def test_eq1_hand_example():
+    """L = 3, one sequence of 6 tokens, 2 heads, M = 3 blocks of 2 tokens: layer 2's means by hand."""
+    counts = np.zeros((3, 2, 6), dtype=np.int32)
+    counts[2, 0] = [1, 2, 3, 4, 5, 6]
+    counts[2, 1] = [0, 0, 1, 1, 10, 0]
+    I = oracle.block_importance(counts, cu_of((6,)), 3)
+    assert np.all(np.isposinf(I[:2]))                       # layers 0 and 1 are always selected
+    np.testing.assert_allclose(I[2], [(1 + 2 + 0 + 0) / 4, (3 + 4 + 1 + 1) / 4, (5 + 6 + 10 + 0) / 4])
+
+
+def test_eq1_mean_over_ragged_sequences_and_mass_invariant():
+    rng = np.random.default_rng(0)
+    lens, L, Hkv, M = (37, 10, 64), 4, 3, 8
+    cu = cu_of(lens)
+    counts = rng.integers(0, 50, size=(L, Hkv, int(cu[-1])), dtype=np.int32)
+    I = oracle.block_importance(counts, cu, M).astype(np.float64)
+    # independent restatement with numpy: block of token t is floor(t*M/N)
+    blk = np.concatenate([np.arange(n) * M // n for n in lens])
+    for l in range(2, L):
+        for m in range(M):
+            sel = counts[l][:, blk == m]
+            assert abs(I[l, m] - sel.mean()) < 1e-5 * max(1.0, sel.mean())
+        entries = np.array([(blk == m).sum() * Hkv for m in range(M)])
+        assert abs((I[l] * entries).sum() - counts[l].sum()) < 1e-3 * counts[l].sum()
+    # uniform counts -> every block has the same importance
+    I = oracle.block_importance(np.full((3, Hkv, int(cu[-1])), 7, dtype=np.int32), cu, M)
+    assert np.all(I[2] == 7.0)
+
+
+def test_eq2_budget_and_clip():
+    L, M = 32, 1024
+    assert oracle.transfer_budget(L, M, 0.5, 1.0) == 1024 * 31 // 2          # M (L-1) T_p / T_t
+    assert oracle.transfer_budget(L, M, 1.0, 6.5) == int(1024 * 31 / 6.5)    # transfer 6.5x the prefill time
+    assert oracle.transfer_budget(L, M, 1e-6, 1.0) == 2 * M                  # clipped from below: two layers always go
+    assert oracle.transfer_budget(L, M, 10.0, 1.0) == L * M                  # low network load: full transfer
+    assert oracle.transfer_budget(L, M, 1.0, 1.0) == M * (L - 1)             # equal times: all but one layer's worth
+
+
+def test_top_kr_always_contains_the_first_two_layers_and_full_budget_is_everything():
+    rng = np.random.default_rng(1)
+    L, M, Hkv = 6, 16, 2
+    cu = cu_of((200,))
+    counts = rng.integers(0, 9, size=(L, Hkv, 200), dtype=np.int32)
+    I = oracle.block_importance(counts, cu, M)
+    for tp in (1e-3, 0.3, 100.0):
+        kr = oracle.transfer_budget(L, M, tp, 1.0)
+        sel = oracle.select_topk(I.reshape(1, 1, L * M), cu_of((L * M,)), cu_of((kr,)))[0, 0]
+        assert set(range(2 * M)) <= set(sel.tolist()) and len(sel) == kr
+        if kr == L * M:
+            assert sel.tolist() == list(range(L * M))
+        rest = np.setdiff1d(np.arange(2 * M, L * M), sel)
+        chosen = np.setdiff1d(sel, np.arange(2 * M))
+        if len(rest) and len(chosen):
+            assert I.ravel()[chosen].min() >= I.ravel()[rest].max()
+
+
+def test_proactive_mask_marks_exactly_the_selected_blocks():
+    lens, M, L = (50, 9), 8, 4
+    cu = cu_of(lens)
+    selected = np.array(sorted([2 * M + 1, 2 * M + 7, 3 * M + 0, 0, 5]), dtype=np.int32)
+    blk = np.concatenate([np.arange(n) * M // n for n in lens])
+    for layer in range(L):
+        mask = oracle.proactive_mask(cu, M, layer, selected)
+        want = np.where(np.isin(layer * M + blk, selected), 1, 2).astype(np.int8)
+        assert np.array_equal(mask, want)
+    assert set(np.unique(oracle.proactive_mask(cu, M, 1, selected)).tolist()) == {2}      # no block of layer 1 selected here
+    full = np.arange(L * M, dtype=np.int32)
+    assert np.all(oracle.proactive_mask(cu, M, 3, full) == 1)                             # full transfer: everything local
