@@ -189,6 +189,35 @@ sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const i
                          void* stream);
 
 /*
+ * Profile-based proactive selection (Section 4.1) -- the second "next" row of the path.
+ *
+ * Blocks: every layer's cache is partitioned along the sequence into M = num_blocks KV blocks; token t of a
+ * sequence of length N_b belongs to block floor(t * M / N_b).  A block holds its tokens' entries of all KV heads.
+ *
+ * sg_profile_accumulate -- S(e), "the number of times entry e is selected in the decoding stage during the
+ *   offline profiling": adds 1 to counts[g][cu[b] + t] for every entry t of one layer's KV index of one decode
+ *   step.  shape->num_layers must be 1; kv_index int32 [H_kv][K_tot] with cu_k as in sg_select_topk;
+ *   counts int32 [H_kv][T] (the caller zeroes it before the first call).  Out-of-range entries set SG_ERR_INDEX.
+ * sg_block_importance -- Eq. 1: importance[l][m] = +inf for l = 0, 1 (the first two layers are always
+ *   selected); otherwise the mean of S(e) over the entries of block B_{l,m} (all its tokens, all KV heads, all
+ *   profiled sequences), a double division rounded to fp32; an empty block gets 0.
+ *   counts int32 [L][H_kv][T]; importance fp32 [L][M].
+ * sg_transfer_budget -- Eq. 2 (host arithmetic, no GPU): K_r = M (L-1) T_p / T_t rounded down, clipped to
+ *   [2M, LM].  The global top-K_r blocks are then sg_select_topk on importance viewed as one row of L*M values.
+ * sg_proactive_mask -- the KV mask of layer `layer` after the proactive transfer (Section 4.2: 1 = locally
+ *   available, 2 = on the remote prefill node): tokens whose block's flat id layer*M + m is in `selected`
+ *   (int32 [num_selected], ascending -- sg_select_topk's output) get 1, all others 2.  kv_mask int8 [T].
+ *   The mask is what sg_split_index consumes.
+ */
+sg_status sg_profile_accumulate(const sg_shape* shape, const int32_t* kv_index, const int32_t* cu_k, int32_t total_sel,
+                                int32_t* counts, int32_t* dev_status, void* stream);
+sg_status sg_block_importance(const sg_shape* shape, const int32_t* counts, int32_t num_blocks, float* importance,
+                              void* stream);
+int64_t sg_transfer_budget(int32_t num_layers, int32_t num_blocks, double t_prefill, double t_transfer);
+sg_status sg_proactive_mask(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
+                            int32_t num_selected, int8_t* kv_mask, void* stream);
+
+/*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.
  *
  * The paper has no counterpart to this call: it computes exactly what sg_score computes.  It exists

@@ -21,7 +21,8 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_score_static", "sg_split_index", "sg_strerror", "sg_last_cuda_error")
+            "sg_score_static", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
+            "sg_transfer_budget", "sg_proactive_mask", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -63,6 +64,14 @@ _lib.sg_select_topk.restype = ctypes.c_int
 _lib.sg_select_topk.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _sz, _vp, _vp]
 _lib.sg_pack_kv.restype = ctypes.c_int
 _lib.sg_pack_kv.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
+_lib.sg_profile_accumulate.restype = ctypes.c_int
+_lib.sg_profile_accumulate.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.sg_block_importance.restype = ctypes.c_int
+_lib.sg_block_importance.argtypes = [_sp, _vp, _i32, _vp, _vp]
+_lib.sg_transfer_budget.restype = ctypes.c_int64
+_lib.sg_transfer_budget.argtypes = [_i32, _i32, ctypes.c_double, ctypes.c_double]
+_lib.sg_proactive_mask.restype = ctypes.c_int
+_lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
 _lib.sg_split_index.restype = ctypes.c_int
 _lib.sg_split_index.argtypes = [_sp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn.restype = ctypes.c_int
@@ -221,3 +230,37 @@ def sg_split_index(shape: Shape, kv_index: torch.Tensor, cu_k: torch.Tensor, tot
                              n_local.data_ptr(), n_remote.data_ptr(), _ptr(dev_status), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_split_index")
+
+
+def sg_profile_accumulate(shape: Shape, kv_index: torch.Tensor, cu_k: torch.Tensor, total_sel: int, counts: torch.Tensor,
+                          dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """S(e) += 1 for every entry of one layer's KV index (counts int32 [H_kv][T], caller-zeroed)."""
+    _check(kv_index, torch.int32, "kv_index"); _check(cu_k, torch.int32, "cu_k"); _check(counts, torch.int32, "counts")
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_profile_accumulate(ctypes.byref(shape), _ptr(kv_index), cu_k.data_ptr(), total_sel, _ptr(counts),
+                                    _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_profile_accumulate")
+
+
+def sg_block_importance(shape: Shape, counts: torch.Tensor, num_blocks: int, importance: torch.Tensor, stream=None) -> None:
+    """Eq. 1: importance fp32 [L][M] from counts int32 [L][H_kv][T]."""
+    _check(counts, torch.int32, "counts"); _check(importance, torch.float32, "importance")
+    rc = _lib.sg_block_importance(ctypes.byref(shape), _ptr(counts), num_blocks, _ptr(importance), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_block_importance")
+
+
+def sg_transfer_budget(num_layers: int, num_blocks: int, t_prefill: float, t_transfer: float) -> int:
+    """Eq. 2: K_r = M (L-1) T_p / T_t, rounded down and clipped to [2M, LM] (host arithmetic)."""
+    return int(_lib.sg_transfer_budget(num_layers, num_blocks, t_prefill, t_transfer))
+
+
+def sg_proactive_mask(shape: Shape, num_blocks: int, layer: int, selected: Optional[torch.Tensor], kv_mask: torch.Tensor,
+                      stream=None) -> None:
+    """KV mask (int8 [T]) of one layer after the proactive transfer: 1 inside the selected blocks, 2 elsewhere."""
+    _check(selected, torch.int32, "selected", True); _check(kv_mask, torch.int8, "kv_mask")
+    n = 0 if selected is None else selected.numel()
+    rc = _lib.sg_proactive_mask(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(kv_mask), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_proactive_mask")
