@@ -196,6 +196,40 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------------------- CUDA arm
 
+def next_rows_timing(dev, cfg, hp, layer=0, reps=20):
+    """Device time of the "next" rows on the workload's shapes: Algorithm 1 (sg_split_index) on one layer's KV
+    index, and the profile chain (sg_profile_accumulate per layer, sg_block_importance, sg_proactive_mask)."""
+    import torch
+    from paper_2607_28150_b200 import binding as sg
+    B, Hkv, T, Ktot, L, M = hp.B, hp.Hkv, hp.T, hp.K_tot, hp.L, 1024
+    gen = torch.Generator(device=dev); gen.manual_seed(77)
+    mask = (torch.randint(0, 100, (T,), generator=gen, device=dev) < 34).to(torch.int8) + 1      # 34 % remote
+    idx = hp.sel_idx[layer].contiguous()
+    re_ = torch.empty_like(idx); loc = torch.empty_like(idx); rem = torch.empty_like(idx)
+    nl = torch.empty((B, Hkv), dtype=torch.int32, device=dev); nr = torch.empty_like(nl)
+    counts = torch.zeros((L, Hkv, T), dtype=torch.int32, device=dev)
+    imp = torch.empty((L, M), dtype=torch.float32, device=dev)
+    pmask = torch.empty(T, dtype=torch.int8, device=dev)
+    selblk = torch.arange(0, 2 * M, dtype=torch.int32, device=dev)
+
+    def timeit(fn):
+        fn(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record(); torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / reps
+
+    return {
+        "split_index_us": timeit(lambda: sg.sg_split_index(hp.shape1, idx, hp.cu_k, Ktot, mask, True, re_, loc, rem, nl, nr)),
+        "profile_accumulate_us_per_layer": timeit(lambda: sg.sg_profile_accumulate(hp.shape1, idx, hp.cu_k, Ktot, counts[layer])),
+        "block_importance_us": timeit(lambda: sg.sg_block_importance(hp.shape, counts, M, imp)),
+        "proactive_mask_us_per_layer": timeit(lambda: sg.sg_proactive_mask(hp.shape1, M, layer, selblk, pmask)),
+        "note": "launch-latency-bound integer kernels (a few KB to a few MB each); eager launches, CUDA events",
+    }
+
+
 def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (128, 1.0, 0.5)), calls=16):
     """sg_sparse_decode_attn alone on points of the decode-heavy sweep (B sequences of 4096 tokens, `sel` of the
     prompt required, `rho` of that index-addressed): the sizes at which the kernel can reach the HBM roofline.
@@ -456,6 +490,7 @@ def run_ours(args):
                "score_tflops": work["score"]["flops"] * fr / t["score"] / 1e12}
 
     kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
+    next_rows = next_rows_timing(dev, cfg, hp) if world == 1 else None
     sweep = None
     if args.workload == "c2" and not args.no_decode_sweep and world == 1:
         del d_k, d_v, h_k, h_v
@@ -477,7 +512,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (3 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "decode_sweep": sweep, "dev_status": status, "setup_s": gen_s,
+        "decode_sweep": sweep, "next_rows": next_rows, "dev_status": status, "setup_s": gen_s,
     }
     print(json.dumps(line))
     if world > 1:
