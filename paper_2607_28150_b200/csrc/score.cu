@@ -75,22 +75,22 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait: gives up after about one second, or as soon as another thread has set *abort_flag.
+// try_wait is given a suspend-time hint, so a waiting thread sleeps in hardware (and is woken when the phase
+// completes) instead of spinning through the issue slots the working warps need.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   uint64_t t0 = 0;
-  for (uint32_t it = 0;; ++it) {
+  for (;;) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(200000u) : "memory");
     if (ok) return true;
     if (*abort_flag) return false;
-    if ((it & 255u) == 255u) {
-      const uint64_t now = global_timer_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > 1000000000ull) { *abort_flag = 1; return false; }
-    }
+    const uint64_t now = global_timer_ns();
+    if (t0 == 0) t0 = now;
+    else if (now - t0 > 1000000000ull) { *abort_flag = 1; return false; }
   }
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
