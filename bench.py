@@ -288,6 +288,9 @@ def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (
 def run_ours(args):
     import torch
     import torch.distributed as dist
+    from paper_2607_28150_b200 import build as _build
+    if not os.path.exists(_build.LIB):
+        _build.build()                                   # in-tree nvcc build; there is no fallback path
     from paper_2607_28150_b200 import binding as sg, workloads as wl
     from paper_2607_28150_b200.pipeline import HotPath
 

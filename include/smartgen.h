@@ -81,7 +81,7 @@ size_t sg_workspace_bytes(int op, const sg_shape* shape, int32_t total_sel, int3
  * q_win       bf16 [L][B][W][H_q][d], dense; row i of sequence b is the query at N_b - W_eff + i.
  * k_cache     bf16, element (l, token, g, c) at l*layer_stride + token*token_stride + g*head_stride + c.
  * importance  fp32 [L][H_kv][T], fully overwritten.
- * Supported: G*W <= 512 (d = 128) or <= 1024 (d = 64), W <= 256.
+ * Supported: G*W <= 512 (d = 128) or <= 1024 (d = 64), W <= 256, B <= 1024; otherwise SG_ERR_UNSUPPORTED.
  */
 sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
                    void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);

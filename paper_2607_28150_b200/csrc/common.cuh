@@ -12,7 +12,7 @@
 namespace sg {
 
 constexpr int kNumSMs = 148;           // B200: 2 dies x 74 SMs; grids are sized in multiples of this
-constexpr int kMaxBatchSmem = 1024;    // prefix arrays longer than this are read from global memory
+constexpr int kMaxBatchSmem = 1024;    // largest batch whose prefix arrays sg_score caches in shared memory
 
 // last failed CUDA call on this host thread (sg_last_cuda_error)
 extern thread_local int g_last_cuda_error;

@@ -27,7 +27,6 @@ constexpr int kDecThreads = 128;
 constexpr int kDecWarps = 4;
 constexpr int kTile = 64;          // tokens per pipeline stage
 constexpr int kStages = 3;
-constexpr int kMaxChunk = 2048;    // tokens per work item in the two-kernel mode
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 

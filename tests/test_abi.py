@@ -58,3 +58,6 @@ def test_host_side_argument_checks_need_no_gpu():
     lib.sg_score.argtypes = sg._lib.sg_score.argtypes
     assert sg.sg_workspace_bytes(sg.SG_OP_SCORE, s) > 16
     assert lib.sg_score(ctypes.byref(s), fake, fake, fake, fake, 16, None, None) == sg.SG_ERR_WORKSPACE
+    # score: more rows per KV head than the shared-memory Q buffer holds is refused, not truncated
+    big = sg.Shape(1, 1, 64, 2, 128, 64, 16384, 16384, 0x1000, 16384 * 256, 256, 128)      # G*W = 2048
+    assert lib.sg_score(ctypes.byref(big), fake, fake, fake, fake, 1 << 30, None, None) == sg.SG_ERR_UNSUPPORTED

@@ -58,6 +58,7 @@ def test_score_llama8b_shape_two_layers():
     ((700,), 1, 5, 6, 2, 64),                          # R = 15: padded to 16 columns
     ((1000, 2000), 1, 24, 16, 2, 128),                 # R = 192: one full and one partial row block
     ((4096,), 1, 8, 32, 2, 64),                        # G = 16, R = 128
+    ((2000, 300), 1, 64, 16, 1, 64),                   # R = 1024 at d = 64: the largest supported row count
 ])
 def test_score_random_shapes(lens, L, W, Hq, Hkv, d):
     run_random(1, lens, L, W, Hq, Hkv, d)
