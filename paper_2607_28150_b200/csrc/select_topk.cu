@@ -253,24 +253,28 @@ __global__ void __launch_bounds__(T) select_topk_reg_kernel(const SelParams p) {
       if (first + e < N && (key[e] & decided) == prefix) atomicAdd(&my_hist[(key[e] >> shift) & (uint32_t)(nbins - 1)], 1u);
     __syncthreads();
     // suffix search: thread t looks at bins nbins-1-t*bpt ... (descending); the bin holding the need-th largest
-    const int bpt = nbins / T > 0 ? nbins / T : 1;
-    uint32_t c[kRegBins / T > 0 ? kRegBins / T : 1];
+    constexpr int kBpt = kRegBins / T;                 // bins per thread in an 11-bit pass (half as many in the 10-bit pass)
+    const int bpt = nbins / T;
+    uint32_t c[kBpt], c2[kBpt];
+    const int bin0 = nbins - 1 - tid * bpt;            // this thread's highest bin; it owns bin0, bin0-1, ...
+#pragma unroll
+    for (int i = 0; i < kBpt; ++i) {                   // all loads first (independent), then the clears for the next pass
+      c[i] = i < bpt ? hist[bin0 - i] : 0u;
+      c2[i] = (i < bpt && copies > 1) ? hist[kRegBins + bin0 - i] : 0u;
+    }
     uint32_t ssum = 0;
 #pragma unroll
-    for (int i = 0; i < (kRegBins / T > 0 ? kRegBins / T : 1); ++i) {
-      const int bin = nbins - 1 - (tid * bpt + i);
-      c[i] = 0;
-      if (i < bpt && bin >= 0) {
-        for (int k = 0; k < copies; ++k) { c[i] += hist[k * kRegBins + bin]; hist[k * kRegBins + bin] = 0; }   // read and clear for the next pass
-      }
+    for (int i = 0; i < kBpt; ++i) {
+      if (i < bpt) { hist[bin0 - i] = 0; if (copies > 1) hist[kRegBins + bin0 - i] = 0; }
+      c[i] += c2[i];
       ssum += c[i];
     }
     const uint32_t exc = block_exclusive_scan<T>(ssum, wsum, lane, warp);   // candidates in bins above this thread's
     if (exc < need && need <= exc + ssum) {
       uint32_t run = exc;
 #pragma unroll
-      for (int i = 0; i < (kRegBins / T > 0 ? kRegBins / T : 1); ++i) {
-        if (run < need && need <= run + c[i]) { sh[0] = (uint32_t)(nbins - 1 - (tid * bpt + i)); sh[1] = need - run; }
+      for (int i = 0; i < kBpt; ++i) {
+        if (run < need && need <= run + c[i]) { sh[0] = (uint32_t)(bin0 - i); sh[1] = need - run; }
         run += c[i];
       }
     }
