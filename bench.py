@@ -7,7 +7,13 @@ One "step" is one pass of the whole path over one batch of synthetic prompts: sg
 sg_select_topk and sg_pack_kv over all layers (one call each), then the workload's decode steps
 (one sg_sparse_decode_attn call per layer per step, replayed from a CUDA graph).  The default
 workload is the Llama-3-8B-shaped cache (32 layers, 8192-token prompt, 10 % budget, 64 decode
-steps).  Rank 0 prints ONE JSON line; see the design doc for the meaning of every key.
+steps).  Rank 0 prints ONE JSON line:
+  value                 (select + pack algorithmic bytes) / (select + pack device time), inputs resident in HBM
+  decode_tokens_per_s   batch * decode steps / decode-stage device time;  stage_ms: every stage of a step
+  e2e                   the same step with host buffers (pinned H2D of caches and queries, D2H of the payload and outputs)
+  roofline / rooflines  per-kernel achieved bytes/s (or flop/s) against the measured copy / bf16 peaks
+  decode_sweep          the decode kernel alone on large-batch points; next_rows: timings of the widened rows
+  cpu_baseline          the CPU oracle timed on a bounded sample of the same workload; clocks: sampled under load
 
 `--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
 """
@@ -31,10 +37,10 @@ if ROOT not in sys.path:
 METRIC = "prefill select+pack GB/s (sparse-decode tokens/s in decode_tokens_per_s)"
 UNIT = "GB/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (bytes; None where no capture exists).  Keyed by workload then kernel.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu --set full captures (bytes; None where no
+# capture exists).  Keyed by workload then kernel.
 NCU_TRAFFIC = {
-    # profiles/kernels_ncu_set_full.md, case A (8 of the 32 layers): per-launch bytes scaled x4 where a launch
+    # captured on 8 of the 32 layers: per-launch bytes scaled x4 where a launch
     # covers all layers; the decode call is per layer.  (pack: its stores were still in L2 when the capture ended.)
     "c2": {"score": 4 * (136.617e6 + 6.328e6), "select": 4 * 2.125e6, "pack": 4 * (27.097e6 + 0.131e6), "decode": 5.163e6},
 }
