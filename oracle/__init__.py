@@ -179,3 +179,10 @@ def proactive_mask(cu_seqlens, num_blocks: int, layer: int, selected) -> np.ndar
     mask = np.zeros(int(cu[-1]), dtype=np.int8)
     _load().sgo_proactive_mask(cu.shape[0] - 1, num_blocks, _p(cu), layer, _p(sel), sel.shape[0], _p(mask))
     return mask
+
+
+def speculative_delivered(num_layers: int, num_blocks: int, k_r: int, ratio: float, iteration: int) -> int:
+    """Blocks on the decode node after `iteration` speculative transfers (Section 4.3)."""
+    lib = _load()
+    lib.sgo_speculative_delivered.restype = ctypes.c_int64
+    return int(lib.sgo_speculative_delivered(num_layers, num_blocks, ctypes.c_int64(k_r), ctypes.c_double(ratio), iteration))

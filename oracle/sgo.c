@@ -399,3 +399,17 @@ int sgo_proactive_mask(int B, int M, const int32_t *cu, int layer, const int32_t
     }
     return 0;
 }
+
+/* Speculative transfer (Section 4.3): after the prefill stage has pushed the top-K_r blocks, every decoding
+ * iteration delivers the next blocks "in the order of their importance, as defined in Eq. 1", at most a fixed
+ * fraction (the speculative ratio) of ALL L*M blocks per iteration.  Number of blocks on the decode node after
+ * `iteration` speculative transfers; the per-iteration quota is ratio * L * M rounded down, at least one block. */
+int64_t sgo_speculative_delivered(int L, int M, int64_t K_r, double ratio, int iteration) {
+    const int64_t total = (int64_t)L * M;
+    int64_t quota = (int64_t)floor(ratio * (double)total);
+    if (quota < 1) quota = 1;
+    int64_t n = K_r + (int64_t)iteration * quota;
+    if (n > total) n = total;
+    if (n < 0) n = 0;
+    return n;
+}

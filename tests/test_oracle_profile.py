@@ -87,3 +87,23 @@ def test_proactive_mask_marks_exactly_the_selected_blocks():
     assert set(np.unique(oracle.proactive_mask(cu, M, 1, selected)).tolist()) == {2}      # no block of layer 1 selected here
     full = np.arange(L * M, dtype=np.int32)
     assert np.all(oracle.proactive_mask(cu, M, 3, full) == 1)                             # full transfer: everything local
+
+
+def test_speculative_schedule_matches_printed_iteration_counts():
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "speculative_iterations.txt")
+    L, M = 40, 1000
+    kr = oracle.transfer_budget(L, M, 1e-9, 1.0)            # minimal proactive transfer: 2M blocks
+    assert kr == 2 * M
+    for line in open(path):
+        if not line.strip() or line.startswith("#"):
+            continue
+        ratio, iters, tol = line.split()
+        it = 0
+        while oracle.speculative_delivered(L, M, kr, float(ratio), it) < L * M:
+            it += 1
+        assert abs(it - int(iters)) <= int(tol)
+    # monotone, starts at K_r, saturates at L*M, at least one block per iteration
+    seq = [oracle.speculative_delivered(L, M, kr, 0.1, i) for i in range(12)]
+    assert seq[0] == kr and seq[-1] == L * M and all(b >= a for a, b in zip(seq, seq[1:]))
+    assert oracle.speculative_delivered(4, 2, 4, 1e-6, 3) == 7
