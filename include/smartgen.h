@@ -208,6 +208,11 @@ sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const i
  *   available, 2 = on the remote prefill node): tokens whose block's flat id layer*M + m is in `selected`
  *   (int32 [num_selected], ascending -- sg_select_topk's output) get 1, all others 2.  kv_mask int8 [T].
  *   The mask is what sg_split_index consumes.
+ * sg_speculative_delivered -- speculative transfer (Section 4.3; host arithmetic, no GPU): after the prefill
+ *   stage pushed the top-K_r blocks, every decoding iteration delivers the next blocks in the order of their
+ *   Eq. 1 importance, at most `ratio` of all L*M blocks per iteration (rounded down, at least one).  Returns the
+ *   number n of blocks on the decode node after `iteration` speculative transfers; the set is the global top-n
+ *   (sg_select_topk with budget n) and the layer masks follow from sg_proactive_mask with that set.
  */
 sg_status sg_profile_accumulate(const sg_shape* shape, const int32_t* kv_index, const int32_t* cu_k, int32_t total_sel,
                                 int32_t* counts, int32_t* dev_status, void* stream);
@@ -216,6 +221,7 @@ sg_status sg_block_importance(const sg_shape* shape, const int32_t* counts, int3
 int64_t sg_transfer_budget(int32_t num_layers, int32_t num_blocks, double t_prefill, double t_transfer);
 sg_status sg_proactive_mask(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
                             int32_t num_selected, int8_t* kv_mask, void* stream);
+int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t k_r, double ratio, int32_t iteration);
 
 /*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.

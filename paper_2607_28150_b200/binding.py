@@ -22,7 +22,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
             "sg_score_static", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
-            "sg_transfer_budget", "sg_proactive_mask", "sg_strerror", "sg_last_cuda_error")
+            "sg_transfer_budget", "sg_proactive_mask", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -70,6 +70,8 @@ _lib.sg_block_importance.restype = ctypes.c_int
 _lib.sg_block_importance.argtypes = [_sp, _vp, _i32, _vp, _vp]
 _lib.sg_transfer_budget.restype = ctypes.c_int64
 _lib.sg_transfer_budget.argtypes = [_i32, _i32, ctypes.c_double, ctypes.c_double]
+_lib.sg_speculative_delivered.restype = ctypes.c_int64
+_lib.sg_speculative_delivered.argtypes = [_i32, _i32, ctypes.c_int64, ctypes.c_double, _i32]
 _lib.sg_proactive_mask.restype = ctypes.c_int
 _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
 _lib.sg_split_index.restype = ctypes.c_int
@@ -264,3 +266,8 @@ def sg_proactive_mask(shape: Shape, num_blocks: int, layer: int, selected: Optio
     rc = _lib.sg_proactive_mask(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(kv_mask), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_proactive_mask")
+
+
+def sg_speculative_delivered(num_layers: int, num_blocks: int, k_r: int, ratio: float, iteration: int) -> int:
+    """Blocks on the decode node after `iteration` speculative transfers of at most `ratio` of all blocks each."""
+    return int(_lib.sg_speculative_delivered(num_layers, num_blocks, k_r, ratio, iteration))

@@ -112,6 +112,17 @@ extern "C" int64_t sg_transfer_budget(int32_t num_layers, int32_t num_blocks, do
   return (int64_t)floor(k);
 }
 
+extern "C" int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t k_r, double ratio,
+                                            int32_t iteration) {
+  const int64_t total = (int64_t)num_layers * num_blocks;
+  int64_t quota = (int64_t)floor(ratio * (double)total);
+  if (quota < 1) quota = 1;
+  int64_t n = k_r + (int64_t)iteration * quota;
+  if (n > total) n = total;
+  if (n < 0) n = 0;
+  return n;
+}
+
 extern "C" sg_status sg_proactive_mask(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
                                        int32_t num_selected, int8_t* kv_mask, void* stream) {
   using namespace sg;

@@ -70,3 +70,40 @@ def test_profile_accumulate_flags_bad_index():
     sg.sg_profile_accumulate(shp, gpu_ops.dev(np.array([[1, 10, 3]], dtype=np.int32)), gpu_ops.dev(ck), 3, counts, st)
     assert gpu_ops.read_status(st) == 1 << sg.SG_ERR_INDEX
     assert counts.cpu().numpy()[0].tolist() == [0, 1, 0, 1, 0, 0, 0, 0, 0, 0]
+
+
+def test_speculative_schedule_masks_grow_until_everything_is_local():
+    """Section 4.3: iteration i has the global top-n_i blocks on the decode node, n_i from the speculative ratio."""
+    import torch
+    import gpu_ops
+    import paper_2607_28150_b200.binding as sg
+    rng = np.random.default_rng(5)
+    L, M, Hkv, lens = 8, 64, 2, (3000, 500)
+    cu = cu_of(lens)
+    T = int(cu[-1])
+    shp1 = gpu_ops.shape_of(1, Hkv, Hkv, 128, 1, cu)
+    I = rng.random((L, M)).astype(np.float32) * 5
+    I[:2] = np.inf
+    kr = sg.sg_transfer_budget(L, M, 0.2, 1.0)
+    prev_local = None
+    it = 0
+    while True:
+        n = sg.sg_speculative_delivered(L, M, kr, 0.10, it)
+        assert n == oracle.speculative_delivered(L, M, kr, 0.10, it)
+        sel_g = gpu_ops.select_topk(I.reshape(1, 1, L * M), cu_of((L * M,)), cu_of((n,)))[0, 0]
+        sel_o = oracle.select_topk(I.reshape(1, 1, L * M), cu_of((L * M,)), cu_of((n,)))[0, 0]
+        assert np.array_equal(sel_g, sel_o)
+        local = np.zeros((L, T), dtype=bool)
+        for l in range(L):
+            m = torch.zeros(T, dtype=torch.int8, device="cuda")
+            sg.sg_proactive_mask(shp1, M, l, gpu_ops.dev(sel_g), m)
+            mg = m.cpu().numpy()
+            assert np.array_equal(mg, oracle.proactive_mask(cu, M, l, sel_o))
+            local[l] = mg == 1
+        if prev_local is not None:
+            assert np.all(local | ~prev_local)                 # nothing that was local becomes remote again
+        prev_local = local
+        if n == L * M:
+            break
+        it += 1
+    assert local.all() and it <= 10                            # 10 % per iteration: complete within 10 iterations
