@@ -135,28 +135,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// Asynchronous TMEM load of 32 consecutive fp32 columns of this thread's lane.  The registers may only be
-// read after tmem_wait_ld() on the same array.
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t (&r)[32], uint32_t taddr) {
+// TMEM load of 32 consecutive fp32 columns of this thread's lane, complete on return (load and wait are one
+// asm statement, so the compiler sees plain outputs).
+__device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-}
-// Wait for this thread's outstanding TMEM loads.  The array is passed in/out so that every later use of its
-// registers depends on this statement.
-__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-      :: "memory");
 }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
@@ -457,8 +448,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
               const int col0 = j * 32;
-              tmem_ld32_issue(cur, t_blk + (uint32_t)col0);
-              tmem_wait_ld(cur);
+              tmem_ld32(cur, t_blk + (uint32_t)col0);
               if (all_visible && row_ok) {
                 float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
                 float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
@@ -573,8 +563,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             for (int j = 0; j < 4; ++j) {
               const int col0 = j * 32;
               if (col0 < ncols) {
-                tmem_ld32_issue(cur, t_blk + (uint32_t)col0);
-                tmem_wait_ld(cur);
+                tmem_ld32(cur, t_blk + (uint32_t)col0);
                 const float* ls = lse2 + blk * 128 + col0;
                 if (all_visible && col0 + 32 <= ncols) {
 #pragma unroll
