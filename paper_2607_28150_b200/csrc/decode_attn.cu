@@ -2,19 +2,22 @@
 //
 // Memory-bound: every attended token costs 2*d*2 bytes of K+V per KV head and only 4*G*d flops.
 // The token list of a (sequence, KV head) -- packed rows first, then local rows addressed through
-// local_idx -- is cut into chunks; one CTA streams one chunk through a 3-stage cp.async ring of
-// 64-token K/V tiles in shared memory (16-byte copies, XOR-swizzled rows so ldmatrix is
-// conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).
-// Each warp owns 16 tokens of a tile: S = Q K^T and O += P V run on bf16 tensor-core MMAs with the
-// G query rows of the KV head padded to 16, the online softmax (base 2) stays in registers.
-// The split-KV partials (m, l, unnormalised O) never leave the chip: the CTAs that share a
-// (sequence, KV head) form a thread-block cluster (1, 2, 4 or 8 CTAs, chosen on the host so that about
-// two CTAs per SM exist and every CTA has at least two tiles); each leaves its partial in its own
-// shared memory and, after a cluster barrier, every CTA merges a slice of the G*d outputs through
-// distributed shared memory with the log-sum-exp rule (m = max m_j, l = sum l_j 2^(m_j-m),
-// o = sum o_j 2^(m_j-m) / l) and writes bf16 out and fp32 lse.  One launch, no workspace.
-// (A two-kernel variant with partials in HBM measured 2x slower on long single-sequence lists and
-// clusters of 16 measured slower than 8 -- few can be co-scheduled -- so neither is kept.)
+// local_idx -- is cut into slices of 16 tokens.  The CTAs that share a (sequence, KV head) split the list
+// evenly; inside a CTA warp w takes slices w, w + warps, ... and streams them through a ring of three
+// K/V slices of its own in shared memory (16-byte cp.async copies, XOR-swizzled rows so ldmatrix is
+// conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).  The ring is
+// private to the warp, so the loop has no block-wide barrier: a warp waits only for its own copies.
+// S = Q K^T and O += P V run on bf16 tensor-core MMAs with the G query rows of the KV head padded to
+// 16; the online softmax (base 2) stays in registers.
+// The split-KV partials (m, l, unnormalised O) never leave the chip: the warps of a CTA merge through
+// shared memory, and the CTAs of a (sequence, KV head) form a thread-block cluster (1, 2, 4 or 8 CTAs);
+// each leaves its partial in its own shared memory and, after a cluster barrier, every CTA merges a
+// slice of the G*d outputs through distributed shared memory with the log-sum-exp rule
+// (m = max m_j, l = sum l_j 2^(m_j-m), o = sum o_j 2^(m_j-m) / l) and writes bf16 out and fp32 lse.
+// One launch, no workspace.
+// (Measured and dropped: a two-kernel variant with partials in HBM, 2x slower on long single-sequence
+// lists; clusters of 16, few of which can be co-scheduled; a block-wide ring of 64-token tiles with a
+// barrier per tile, 10-25 % slower at every size.)
 // The launch uses programmatic dependent launch, so back-to-back decode calls overlap their launch
 // latency and prologue with the previous call's tail.
 #include "common.cuh"
@@ -23,10 +26,7 @@
 namespace sg {
 namespace {
 
-constexpr int kDecThreads = 128;
-constexpr int kDecWarps = 4;
-constexpr int kTile = 64;          // tokens per pipeline stage
-constexpr int kStages = 3;
+constexpr int kSlice = 16;         // tokens per warp step (one m16n8k16 k-extent of P V)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -91,16 +91,19 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // kHi: the KV head has more than 8 query rows, so MMA rows 8..15 carry data too.
-template <int D, bool kHi>
-__global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const DecParams p) {
+// kDecWarps warps per CTA, each with a private ring of kBuf slices: (8, 3) gives one CTA per SM, (4, 3) two.
+template <int D, bool kHi, int kDecWarps, int kBuf>
+__global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode_partial_kernel(const DecParams p) {
+  constexpr int kDecThreads = kDecWarps * 32;
   constexpr int kRowBytes = D * 2;
   constexpr int kChunksPerRow = D / 8;                       // 16-byte chunks
-  constexpr int kTileBytes = kTile * kRowBytes;
-  constexpr int kCopiesPerThread = kTile * kChunksPerRow / kDecThreads;
+  constexpr int kSliceBytes = kSlice * kRowBytes;            // K (or V) rows of one slice
+  constexpr int kCopiesPerLane = kSlice * kChunksPerRow / 32;
+  constexpr uint32_t kFull = 0xffffffffu;
   extern __shared__ __align__(128) uint8_t smem_raw[];
-  uint8_t* sk = smem_raw;                                    // [kStages][kTile][D] bf16, swizzled
-  uint8_t* sv = smem_raw + kStages * kTileBytes;
-  uint8_t* s_valid = smem_raw + 2 * kStages * kTileBytes;    // [kStages][kTile] 1 = row holds a real token
+  // per warp: kBuf slices of K, then kBuf slices of V, rows XOR-swizzled; after all rings one validity
+  // word per (warp, buffer)
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(smem_raw + kDecWarps * kBuf * 2 * kSliceBytes);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
@@ -112,7 +115,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   const int c0 = p.cu[b];
   const int nseq = p.cu[b + 1] - c0;
   // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
-  const int span = ((((kb + nl + p.csize - 1) / p.csize) + kTile - 1) / kTile) * kTile;
+  const int span = ((((kb + nl + p.csize - 1) / p.csize) + kSlice - 1) / kSlice) * kSlice;
   const int range_beg = min(kb + nl, c * span);
   const int range_end = min(kb + nl, range_beg + span);
 
@@ -120,28 +123,38 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   const uint16_t* pv_base = p.packed_v + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
   const uint16_t* lk_base = p.local_k + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
   const uint16_t* lv_base = p.local_v + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
-  const uint32_t sk_u32 = smem_u32(sk), sv_u32 = smem_u32(sv);
+  const uint32_t wk_u32 = smem_u32(smem_raw) + warp * (kBuf * 2 * kSliceBytes);   // this warp's K ring
+  const uint32_t wv_u32 = wk_u32 + kBuf * kSliceBytes;                            // and its V ring
 
   const int pos_beg = range_beg, ntok = range_end - range_beg;
-  const int ntiles = (ntok + kTile - 1) / kTile;
+  const int nslices = (ntok + kSlice - 1) / kSlice;
+  // warp w streams slices w, w + kDecWarps, ... of the range, so the CTA walks memory front to back
+  const int nmine = nslices > warp ? (nslices - warp + kDecWarps - 1) / kDecWarps : 0;
   const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] - kb;   // indexed by list position
-  // Local indices of the rows this thread copies in `tile` (read one tile ahead of their use).
-  auto fetch_idx = [&](int tile, int (&idx)[kCopiesPerThread]) {
-#pragma unroll
-    for (int i = 0; i < kCopiesPerThread; ++i) {
-      const int li = tile * kTile + (tid + i * kDecThreads) / kChunksPerRow;
-      const int pos = pos_beg + li;
-      idx[i] = (li < ntok && pos >= kb) ? __ldg(idx_base + pos) : 0;
-    }
+  // Lane r (and r + 16) holds the local index of row r of the warp's j-th slice, read one slice ahead.
+  auto fetch_idx = [&](int j) -> int {
+    const int li = (warp + j * kDecWarps) * kSlice + (lane & 15);
+    const int pos = pos_beg + li;
+    return (j < nmine && li < ntok && pos >= kb) ? __ldg(idx_base + pos) : 0;
   };
-  auto load_tile = [&](int tile, int stage, const int (&idx)[kCopiesPerThread]) {
+  auto load_slice = [&](int j, int buf, int idx_reg) {
+    const int li0 = (warp + j * kDecWarps) * kSlice;
+    {
+      const int li = li0 + (lane & 15), pos = pos_beg + li;
+      const bool in_list = li < ntok;
+      const bool ok = in_list && (pos < kb || (idx_reg >= 0 && idx_reg < nseq));
+      if (in_list && !ok && lane < 16) raise(p.dev_status, SG_ERR_INDEX);
+      const uint32_t mask = __ballot_sync(kFull, ok) & 0xffffu;
+      if (lane == 0) s_mask[warp * kBuf + buf] = mask;        // bit r: row r holds a real token
+    }
 #pragma unroll
-    for (int i = 0; i < kCopiesPerThread; ++i) {
-      const int qid = tid + i * kDecThreads;
+    for (int i = 0; i < kCopiesPerLane; ++i) {
+      const int qid = lane + i * 32;
       const int row = qid / kChunksPerRow;
       const int col = qid % kChunksPerRow;
-      const int li = tile * kTile + row;                      // index within this CTA's range
+      const int li = li0 + row;
       const int pos = pos_beg + li;
+      const int t = __shfl_sync(kFull, idx_reg, row);
       const uint16_t* srck = p.packed_k;
       const uint16_t* srcv = p.packed_v;
       int bytes = 0;
@@ -150,21 +163,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
           srck = pk_base + (int64_t)pos * D + col * 8;
           srcv = pv_base + (int64_t)pos * D + col * 8;
           bytes = 16;
-        } else {
-          const int t = idx[i];
-          if (t >= 0 && t < nseq) {
-            srck = lk_base + (int64_t)t * p.ts + col * 8;
-            srcv = lv_base + (int64_t)t * p.ts + col * 8;
-            bytes = 16;
-          } else if (col == 0) {
-            raise(p.dev_status, SG_ERR_INDEX);
-          }
+        } else if (t >= 0 && t < nseq) {
+          srck = lk_base + (int64_t)t * p.ts + col * 8;
+          srcv = lv_base + (int64_t)t * p.ts + col * 8;
+          bytes = 16;
         }
       }
-      const uint32_t off = stage * kTileBytes + row * kRowBytes + ((col ^ (row & 7)) << 4);
-      cp_async16(sk_u32 + off, srck, bytes);                  // bytes == 0 zero-fills the row
-      cp_async16(sv_u32 + off, srcv, bytes);
-      if (col == 0) s_valid[stage * kTile + row] = bytes ? 1 : 0;
+      const uint32_t off = buf * kSliceBytes + row * kRowBytes + ((col ^ (row & 7)) << 4);
+      cp_async16(wk_u32 + off, srck, bytes);                  // bytes == 0 zero-fills the row
+      cp_async16(wv_u32 + off, srcv, bytes);
     }
   };
 
@@ -173,15 +180,15 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   for (int i = 0; i < D / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
-  int idx_next[kCopiesPerThread];
+  int idx_next;
   {
-    int idx_pro[kStages - 1][kCopiesPerThread];
+    int idx_pro[kBuf - 1];
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) fetch_idx(s, idx_pro[s]);
-    fetch_idx(kStages - 1, idx_next);
+    for (int s = 0; s < kBuf - 1; ++s) idx_pro[s] = fetch_idx(s);
+    idx_next = fetch_idx(kBuf - 1);
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) {
-      if (s < ntiles) load_tile(s, s, idx_pro[s]);
+    for (int s = 0; s < kBuf - 1; ++s) {
+      if (s < nmine) load_slice(s, s, idx_pro[s]);
       cp_async_commit();
     }
   }
@@ -204,21 +211,22 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     }
   }
 
+  // The ring is private to the warp: no block-wide barrier inside the loop, the warps drift freely.
 #pragma unroll 1
-  for (int tile = 0; tile < ntiles; ++tile) {
-    cp_async_wait<kStages - 2>();
-    __syncthreads();
+  for (int j = 0; j < nmine; ++j) {
+    cp_async_wait<kBuf - 2>();
+    __syncwarp();
     {
-      const int nt = tile + kStages - 1;
-      if (nt < ntiles) load_tile(nt, nt % kStages, idx_next);
+      const int nj = j + kBuf - 1;
+      if (nj < nmine) load_slice(nj, nj % kBuf, idx_next);
       cp_async_commit();
-      fetch_idx(nt + 1, idx_next);
+      idx_next = fetch_idx(nj + 1);
     }
-    const int stage = tile % kStages;
-    const uint32_t k_st = sk_u32 + stage * kTileBytes;
-    const uint32_t v_st = sv_u32 + stage * kTileBytes;
-    const int wrow = warp * 16;
-    if (tile * kTile + wrow >= ntok) continue;               // this warp's 16 tokens are all padding
+    const int buf = j % kBuf;
+    const uint32_t k_st = wk_u32 + buf * kSliceBytes;
+    const uint32_t v_st = wv_u32 + buf * kSliceBytes;
+    const uint32_t vmask = s_mask[warp * kBuf + buf];
+    constexpr int wrow = 0;
 
     // S = Q K^T for 16 tokens (two n8 tiles)
     float s_acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -240,7 +248,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
     for (int j = 0; j < 2; ++j) {
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const bool valid = s_valid[stage * kTile + wrow + j * 8 + 2 * (lane & 3) + e] != 0;
+        const bool valid = (vmask >> (j * 8 + 2 * (lane & 3) + e)) & 1u;
         s_acc[j][e] = valid ? s_acc[j][e] * p.scale_log2 : -INFINITY;
         mx_lo = fmaxf(mx_lo, s_acc[j][e]);
         if (kHi) {
@@ -312,7 +320,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   cp_async_wait<0>();
   __syncthreads();
 
-  // merge the four warps through shared memory (the pipeline buffers are free now)
+  // merge the warps through shared memory (the rings are free now)
   float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
   float* sm_m = sm_o + kDecWarps * 16 * D;                    // [kDecWarps][16]
   float* sm_l = sm_m + kDecWarps * 16;
@@ -384,20 +392,36 @@ __global__ void __launch_bounds__(kDecThreads, 2) decode_partial_kernel(const De
   }
 }
 
-template <int D>
-constexpr int decode_smem_bytes() { return 2 * kStages * kTile * D * 2 + kStages * kTile; }
+template <int D, int kDecWarps, int kBuf>
+constexpr int decode_smem_bytes() { return kDecWarps * kBuf * 2 * kSlice * D * 2 + kDecWarps * kBuf * 4; }
 
 }  // namespace
 
-// CTAs per (sequence, KV head) = cluster size: a power of two <= 8 (the portable cluster limit).
-int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_loc) {
+// Launch shape, from what a sweep over batch sizes and list lengths measured.  CTAs beyond one wave
+// of resident CTAs never paid, so a (sequence, KV head) pair is split over a cluster only while all
+// clusters fit on the SMs at one CTA each.
+//  * pairs <= SMs: warps = 8, one CTA per SM; csize = the cluster size (a power of two <= 8, the
+//    portable limit) that gives each warp about one slice, capped by the SM count (12 warps per CTA
+//    measured slower than 8: the merge grows faster than the streaming shrinks);
+//  * more pairs: csize = 1 and warps = 4, two CTAs per SM, so that one CTA's prologue and merge overlap
+//    the other's streaming -- except long lists whose CTA count fills waves of one CTA per SM better.
+void decode_plan(const sg_shape* shape, int32_t total_sel, int32_t total_loc, int* csize, int* warps) {
   const int64_t pairs = (int64_t)shape->batch * shape->num_kv_heads;
-  const int64_t avg_tiles = (((int64_t)total_sel + total_loc) / shape->batch + kTile - 1) / kTile;
-  int by_work = 1;
-  while (by_work < 8 && by_work * 2 * 2 <= avg_tiles) by_work *= 2;        // at least two tiles per CTA
-  int by_fill = 1;
-  while (by_fill < 8 && pairs * by_fill < 2 * kNumSMs) by_fill *= 2;        // about two CTAs per SM
-  return by_work < by_fill ? by_work : by_fill;
+  const int64_t avg_tokens = ((int64_t)total_sel + total_loc) / shape->batch;
+  int W = 4, cs = 1;
+  if (pairs <= kNumSMs) {
+    W = 8;
+    int fit = 1;
+    while (fit < 8 && pairs * fit * 2 <= kNumSMs) fit *= 2;
+    int work = 1;
+    while (work < 8 && (int64_t)work * W * kSlice < avg_tokens) work *= 2;
+    cs = fit < work ? fit : work;
+  } else {
+    auto fill = [&](int64_t slots) { return (double)pairs / (double)(((pairs + slots - 1) / slots) * slots); };
+    W = (avg_tokens >= 1024 && fill(kNumSMs) > fill(2 * kNumSMs) + 0.05) ? 8 : 4;
+  }
+  *csize = cs;
+  *warps = W;
 }
 
 size_t decode_workspace_bytes(const sg_shape*, int32_t, int32_t) { return 0; }   // partials stay on chip
@@ -446,7 +470,8 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.G = G;
   p.K_tot = total_sel;
   p.NL_tot = total_loc;
-  p.csize = decode_cluster_size(shape, total_sel, total_loc);
+  int warps = 4;
+  decode_plan(shape, total_sel, total_loc, &p.csize, &warps);
   p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
   const int64_t grid_x = (int64_t)shape->batch * p.csize;
   if (grid_x > 0x7fffffffLL || shape->num_kv_heads > 65535) return SG_ERR_UNSUPPORTED;
@@ -462,17 +487,23 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   cfg.stream = static_cast<cudaStream_t>(stream);
   cfg.attrs = attrs;
   cfg.numAttrs = p.csize > 1 ? 2 : 1;
-  cfg.blockDim = dim3(kDecThreads);
+  cfg.blockDim = dim3((unsigned)warps * 32);
   // one launch: sequences with empty lists still get out = 0 and lse = -inf
   cfg.gridDim = dim3((unsigned)grid_x, (unsigned)shape->num_kv_heads);
-#define SG_LAUNCH_DECODE(DD, HI)                                                          \
-  do {                                                                                    \
-    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI>), decode_smem_bytes<DD>());             \
-    cfg.dynamicSmemBytes = decode_smem_bytes<DD>();                                       \
-    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<DD, HI>, p));              \
+#define SG_LAUNCH_DECODE(DD, HI, WW, BB)                                                      \
+  do {                                                                                        \
+    SG_ENSURE_SMEM((decode_partial_kernel<DD, HI, WW, BB>), (decode_smem_bytes<DD, WW, BB>())); \
+    cfg.dynamicSmemBytes = decode_smem_bytes<DD, WW, BB>();                                   \
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_partial_kernel<DD, HI, WW, BB>, p));          \
   } while (0)
-  if (D == 128) { if (G > 8) SG_LAUNCH_DECODE(128, true); else SG_LAUNCH_DECODE(128, false); }
-  else          { if (G > 8) SG_LAUNCH_DECODE(64, true);  else SG_LAUNCH_DECODE(64, false); }
+#define SG_LAUNCH_DECODE_W(DD, HI)                         \
+  do {                                                     \
+    if (warps == 8) SG_LAUNCH_DECODE(DD, HI, 8, 3);        \
+    else SG_LAUNCH_DECODE(DD, HI, 4, 3);                   \
+  } while (0)
+  if (D == 128) { if (G > 8) SG_LAUNCH_DECODE_W(128, true); else SG_LAUNCH_DECODE_W(128, false); }
+  else          { if (G > 8) SG_LAUNCH_DECODE_W(64, true);  else SG_LAUNCH_DECODE_W(64, false); }
+#undef SG_LAUNCH_DECODE_W
 #undef SG_LAUNCH_DECODE
   return SG_OK;
 }

@@ -9,5 +9,5 @@ namespace sg {
 size_t score_workspace_bytes(const sg_shape* shape);
 size_t decode_workspace_bytes(const sg_shape* shape, int32_t total_sel, int32_t total_loc);
 // Cluster size (CTAs per sequence and KV head) the decode kernel uses for a call of this size.
-int decode_cluster_size(const sg_shape* shape, int32_t total_sel, int32_t total_loc);
+void decode_plan(const sg_shape* shape, int32_t total_sel, int32_t total_loc, int* csize, int* warps);
 }  // namespace sg

@@ -47,9 +47,11 @@ def compare(args, **kw):
     ((4096,) * 3, (100, 4096, 1), (3996, 0, 0), 8, 8, 128),   # G = 1, full budget, single token
     ((2000,), (333,), (100,), 32, 2, 128),                    # G = 16
     ((513,), (65,), (63,), 16, 2, 64),                        # G = 8, d = 64, ragged tiles
-    ((12000,), (5000,), (3333,), 8, 2, 128),                  # few heads, long lists: two-kernel split-KV mode
-    ((9000, 100), (4100, 10), (4500, 90), 4, 1, 128),         # two-kernel mode, ragged
-    ((25000,) * 3, (12000,) * 3, (8000,) * 3, 8, 8, 128),     # cluster mode, CTA ranges longer than the index staging buffer
+    ((12000,), (5000,), (3333,), 8, 2, 128),                  # few heads, long lists: clusters of 8, many slices per warp
+    ((9000, 100), (4100, 10), (4500, 90), 4, 1, 128),         # one head, ragged pair of sequences
+    ((25000,) * 3, (12000,) * 3, (8000,) * 3, 8, 8, 128),     # clusters of 4, long CTA ranges
+    (tuple(200 + 13 * i for i in range(40)), tuple(5 * i for i in range(40)), tuple(150 - 3 * i for i in range(40)), 32, 8, 128),   # more pairs than SMs: 4-warp CTAs, no clusters
+    (tuple(90 + 7 * i for i in range(80)), (33,) * 80, tuple(i % 50 for i in range(80)), 32, 2, 64),   # same, G = 16, d = 64
 ])
 def test_decode_matches_oracle(lens, ks, nls, Hq, Hkv, d):
     compare(build(0, lens, ks, nls, Hq, Hkv, d))
