@@ -78,12 +78,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
-__device__ __forceinline__ float ld_dsmem_f32(const float* local_ptr, uint32_t cta_rank) {
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void st_dsmem_f32(float* local_ptr, uint32_t cta_rank, float v) {
   uint32_t remote;
-  float v;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
-  asm volatile("ld.shared::cluster.f32 %0, [%1];\n" : "=f"(v) : "r"(remote) : "memory");
-  return v;
+  asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(remote), "f"(v) : "memory");
 }
 // Programmatic dependent launch: let the next kernel in the stream start its prologue now, and wait
 // for the previous kernel's memory before touching anything it may have written.
@@ -104,10 +106,16 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   // per warp: kBuf slices of K, then kBuf slices of V, rows XOR-swizzled; after all rings one validity
   // word per (warp, buffer)
   uint32_t* s_mask = reinterpret_cast<uint32_t*>(smem_raw + kDecWarps * kBuf * 2 * kSliceBytes);
+  // Receive area for the cluster merge, never aliased by the rings: the slice of the G*d outputs this CTA
+  // owns, as every rank's partial: rx_o [8][per], rx_m [8][16], rx_l [8][16].
+  float* rx_m = reinterpret_cast<float*>(s_mask + kDecWarps * kBuf);
+  float* rx_l = rx_m + 8 * 16;
+  float* rx_o = rx_l + 8 * 16;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
   pdl_launch_dependents();
+  if (p.csize > 1) cluster_arrive_relaxed();                   // "this CTA runs": awaited before the first remote store
   const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
   const int kb = p.cu_k[b + 1] - p.cu_k[b];
@@ -324,21 +332,26 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
   float* sm_m = sm_o + kDecWarps * 16 * D;                    // [kDecWarps][16]
   float* sm_l = sm_m + kDecWarps * 16;
+  const bool w_lo = r_lo < p.G, w_hi = kHi && r_hi < p.G;      // rows >= G are padding and never read
   if ((lane & 3) == 0) {
-    sm_m[warp * 16 + r_lo] = m_lo; sm_l[warp * 16 + r_lo] = l_lo;
-    sm_m[warp * 16 + r_hi] = kHi ? m_hi : -INFINITY; sm_l[warp * 16 + r_hi] = kHi ? l_hi : 0.f;
+    if (w_lo) { sm_m[warp * 16 + r_lo] = m_lo; sm_l[warp * 16 + r_lo] = l_lo; }
+    if (w_hi) { sm_m[warp * 16 + r_hi] = m_hi; sm_l[warp * 16 + r_hi] = l_hi; }
   }
 #pragma unroll
   for (int i = 0; i < D / 8; ++i) {
     const int col = i * 8 + 2 * (lane & 3);
     float* dst = sm_o + (warp * 16 + r_lo) * D + col;
-    dst[0] = o_acc[i][0]; dst[1] = o_acc[i][1];
-    if (kHi) { dst[8 * D] = o_acc[i][2]; dst[8 * D + 1] = o_acc[i][3]; }
+    if (w_lo) *reinterpret_cast<float2*>(dst) = make_float2(o_acc[i][0], o_acc[i][1]);
+    if (w_hi) *reinterpret_cast<float2*>(dst + 8 * D) = make_float2(o_acc[i][2], o_acc[i][3]);
   }
   __syncthreads();
-  float* sm_co = sm_l + kDecWarps * 16;                       // CTA-level partial: O [16][D], m [16], l [16]
-  float* sm_cm = sm_co + 16 * D;
-  float* sm_cl = sm_cm + 16;
+  // CTA-level partial of every output; with a cluster, each rank owns a slice of the G*d outputs and
+  // every CTA pushes its partial of a slice into the owner's receive area (distributed shared memory).
+  const int cs = p.csize;
+  const int per = (p.G * D + cs - 1) / cs;
+  __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
+  float* lsep = p.lse ? p.lse + (int64_t)b * p.Hq + (int64_t)g * p.G : nullptr;
+  if (cs > 1) cluster_wait();                                  // every CTA of the cluster has started
   for (int e = tid; e < p.G * D; e += kDecThreads) {
     const int r = e / D, col = e - r * D;
     float M = -INFINITY;
@@ -352,27 +365,29 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       L += sm_l[w * 16 + r] * f;
       O += sm_o[(w * 16 + r) * D + col] * f;
     }
-    sm_co[e] = O;
-    if (col == 0) { sm_cm[r] = M; sm_cl[r] = L; }
+    if (cs == 1) {
+      outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+      if (lsep && col == 0) lsep[r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+    } else {
+      const int owner = e / per;
+      st_dsmem_f32(rx_o + c * per + (e - owner * per), owner, O);
+      if (col == 0) {
+        for (int j = 0; j < cs; ++j) { st_dsmem_f32(rx_m + c * 16 + r, j, M); st_dsmem_f32(rx_l + c * 16 + r, j, L); }
+      }
+    }
   }
-  {
-    // Every CTA of the cluster merges a slice of the G*D outputs, reading all ranks' partials.
-    const int cs = p.csize;
-    if (cs > 1) cluster_sync_all(); else __syncthreads();
-    const int per = (p.G * D + cs - 1) / cs;
+  if (cs > 1) {
+    cluster_sync_all();                                       // release the pushes, acquire everyone else's
     const int e_beg = c * per, e_end = min(p.G * D, e_beg + per);
-    __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
     for (int e = e_beg + tid; e < e_end; e += kDecThreads) {
       const int r = e / D, col = e - r * D;
-      float mj[8], lj[8], oj[8];                             // all ranks' partials, loaded independently
+      float mj[8], lj[8], oj[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        mj[j] = -INFINITY; lj[j] = 0.f; oj[j] = 0.f;
-        if (j < cs) {
-          mj[j] = cs > 1 ? ld_dsmem_f32(sm_cm + r, j) : sm_cm[r];
-          lj[j] = cs > 1 ? ld_dsmem_f32(sm_cl + r, j) : sm_cl[r];
-          oj[j] = cs > 1 ? ld_dsmem_f32(sm_co + e, j) : sm_co[e];
-        }
+        const bool on = j < cs;
+        mj[j] = on ? rx_m[j * 16 + r] : -INFINITY;
+        lj[j] = on ? rx_l[j * 16 + r] : 0.f;
+        oj[j] = on ? rx_o[j * per + (e - e_beg)] : 0.f;
       }
       float M = -INFINITY;
 #pragma unroll
@@ -386,14 +401,16 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
         O += oj[j] * f;
       }
       outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
-      if (p.lse && col == 0) p.lse[(int64_t)b * p.Hq + (int64_t)g * p.G + r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
+      if (lsep && col == 0) lsep[r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     }
-    if (cs > 1) cluster_sync_all();                           // keep every CTA's shared memory alive until all reads are done
+    // no trailing barrier: after the one above nobody touches another CTA's shared memory
   }
 }
 
 template <int D, int kDecWarps, int kBuf>
-constexpr int decode_smem_bytes() { return kDecWarps * kBuf * 2 * kSlice * D * 2 + kDecWarps * kBuf * 4; }
+constexpr int decode_smem_bytes() {
+  return kDecWarps * kBuf * 2 * kSlice * D * 2 + kDecWarps * kBuf * 4 + (2 * 8 * 16 + 16 * D) * 4;   // rings, masks, receive area
+}
 
 }  // namespace
 
