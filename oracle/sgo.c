@@ -413,3 +413,30 @@ int64_t sgo_speculative_delivered(int L, int M, int64_t K_r, double ratio, int i
     if (n < 0) n = 0;
     return n;
 }
+
+/* Online proactive transfer of one layer (Section 4.1, "Online KV transfer"): the layer's cache is split into
+ * M blocks; every block whose position is among the top-K_r (flat id layer*M + m in `selected`) is written,
+ * all KV heads, K and V, to the same token positions of the decode-side cache; nothing else is written.
+ * Caches of this layer: uint16 [T][Hkv][d] (dense).  selected int32 [K_r], any order. */
+int sgo_push_blocks(int B, int Hkv, int d, int M, const int32_t *cu, int layer, const int32_t *selected, int K_r,
+                    const uint16_t *src_k, const uint16_t *src_v, uint16_t *dst_k, uint16_t *dst_v) {
+    for (int b = 0; b < B; ++b) {
+        const int64_t N = cu[b + 1] - cu[b];
+        for (int m = 0; m < M; ++m) {
+            const int32_t id = (int32_t)((int64_t)layer * M + m);
+            int pushed = 0;
+            for (int j = 0; j < K_r; ++j)
+                if (selected[j] == id) { pushed = 1; break; }
+            if (!pushed) continue;
+            for (int64_t t = 0; t < N; ++t) {
+                if (block_of(t, N, M) != m) continue;      /* E(B_{l,m}): the tokens of the block */
+                const int64_t row = (cu[b] + t) * Hkv * (int64_t)d;
+                for (int64_t e = 0; e < (int64_t)Hkv * d; ++e) {
+                    dst_k[row + e] = src_k[row + e];
+                    dst_v[row + e] = src_v[row + e];
+                }
+            }
+        }
+    }
+    return 0;
+}

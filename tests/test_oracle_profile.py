@@ -107,3 +107,61 @@ def test_speculative_schedule_matches_printed_iteration_counts():
     seq = [oracle.speculative_delivered(L, M, kr, 0.1, i) for i in range(12)]
     assert seq[0] == kr and seq[-1] == L * M and all(b >= a for a, b in zip(seq, seq[1:]))
     assert oracle.speculative_delivered(4, 2, 4, 1e-6, 3) == 7
+
+
+def _caches(seed, lens, Hkv, d):
+    rng = np.random.default_rng(seed)
+    T = int(sum(lens))
+    mk = lambda: rng.integers(0, 1 << 16, size=(T, Hkv, d), dtype=np.uint16)
+    return mk(), mk(), mk(), mk()
+
+
+def test_push_blocks_hand_example():
+    """Section 4.1, online transfer: 10 tokens in M = 4 blocks are {0,1,2} {3,4} {5,6,7} {8,9} (token t is in block
+    floor(t M / N)); pushing blocks 1 and 3 of layer 2 moves rows 3, 4, 8, 9 and nothing else."""
+    sk, sv, dk, dv = _caches(0, (10,), 2, 8)
+    M, layer = 4, 2
+    gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu_of((10,)), M, layer, np.array([0, 5, layer * M + 1, layer * M + 3, 13], dtype=np.int32))
+    moved = np.array([3, 4, 8, 9])
+    kept = np.array([0, 1, 2, 5, 6, 7])
+    assert np.array_equal(gk[moved], sk[moved]) and np.array_equal(gv[moved], sv[moved])
+    assert np.array_equal(gk[kept], dk[kept]) and np.array_equal(gv[kept], dv[kept])
+
+
+def test_push_blocks_agrees_with_the_kv_mask_and_covers_all_heads():
+    """The pushed rows are exactly the rows the proactive KV mask marks local (1); rows marked remote (2) keep the
+    destination's old bytes; K and V, every head, every element of a pushed row."""
+    lens = (37, 5, 64, 1)
+    cu = cu_of(lens)
+    M, L = 8, 5
+    rng = np.random.default_rng(3)
+    selected = np.sort(rng.choice(L * M, size=17, replace=False)).astype(np.int32)
+    sk, sv, dk, dv = _caches(1, lens, 3, 16)
+    for layer in range(L):
+        gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu, M, layer, selected)
+        local = oracle.proactive_mask(cu, M, layer, selected) == 1
+        blk = np.concatenate([np.arange(n) * M // n for n in lens])         # independent block geometry
+        assert np.array_equal(local, np.isin(layer * M + blk, selected))
+        assert np.array_equal(gk, np.where(local[:, None, None], sk, dk))
+        assert np.array_equal(gv, np.where(local[:, None, None], sv, dv))
+
+
+def test_push_blocks_all_and_none():
+    lens = (20, 33)
+    cu = cu_of(lens)
+    sk, sv, dk, dv = _caches(2, lens, 2, 8)
+    M = 6
+    gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu, M, 1, np.arange(M, 2 * M, dtype=np.int32))
+    assert np.array_equal(gk, sk) and np.array_equal(gv, sv)
+    gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu, M, 1, np.arange(0, M, dtype=np.int32))     # another layer's blocks
+    assert np.array_equal(gk, dk) and np.array_equal(gv, dv)
+    gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu, M, 0, np.zeros(0, dtype=np.int32))
+    assert np.array_equal(gk, dk) and np.array_equal(gv, dv)
+
+
+def test_push_blocks_more_blocks_than_tokens():
+    """M > N: most blocks are empty, every token is alone in its block floor(t M / N)."""
+    sk, sv, dk, dv = _caches(4, (3,), 1, 8)
+    gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu_of((3,)), 8, 0, np.array([2, 3], dtype=np.int32))   # token 1 -> block 2
+    assert np.array_equal(gk[1], sk[1]) and np.array_equal(gk[[0, 2]], dk[[0, 2]])
+    assert np.array_equal(gv[1], sv[1]) and np.array_equal(gv[[0, 2]], dv[[0, 2]])
