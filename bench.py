@@ -202,7 +202,7 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------------------- CUDA arm
 
-def next_rows_timing(dev, cfg, hp, layer=0, reps=20):
+def next_rows_timing(dev, cfg, hp, k_cache, v_cache, layer=0, reps=20):
     """Device time of the "next" rows on the workload's shapes: Algorithm 1 (sg_split_index) on one layer's KV
     index, and the profile chain (sg_profile_accumulate per layer, sg_block_importance, sg_proactive_mask)."""
     import torch
@@ -217,6 +217,18 @@ def next_rows_timing(dev, cfg, hp, layer=0, reps=20):
     imp = torch.empty((L, M), dtype=torch.float32, device=dev)
     pmask = torch.empty(T, dtype=torch.int8, device=dev)
     selblk = torch.arange(0, 2 * M, dtype=torch.int32, device=dev)
+    # block push: every block of one layer (Eq. 1 always selects layers 0 and 1), rotating over the layers so the
+    # source is not L2-resident; one layer of K+V read and written per call
+    dst_k = torch.empty_like(k_cache[0]); dst_v = torch.empty_like(v_cache[0])
+    push_sel = [torch.arange(l * M, (l + 1) * M, dtype=torch.int32, device=dev) for l in range(L)]
+
+    def push_all_layers():                                   # L calls, one per layer, replayed from a CUDA graph
+        for l in range(L):
+            sg.sg_push_blocks(hp.shape1, M, l, push_sel[l], k_cache[l], v_cache[l], dst_k, dst_v)
+    push_bytes = 2 * 2 * T * Hkv * hp.d * 2
+    dst_all_k = torch.empty_like(k_cache); dst_all_v = torch.empty_like(v_cache)
+    sel_all = torch.arange(0, L * M, dtype=torch.int32, device=dev)
+    sel_40 = torch.arange(0, L * M, dtype=torch.int32, device=dev)[torch.randperm(L * M, generator=gen, device=dev)[: (2 * L * M) // 5]].sort().values.contiguous()
 
     def timeit(fn):
         fn(); torch.cuda.synchronize()
@@ -227,12 +239,32 @@ def next_rows_timing(dev, cfg, hp, layer=0, reps=20):
         e1.record(); torch.cuda.synchronize()
         return 1e3 * e0.elapsed_time(e1) / reps
 
+    def timeit_graph(fn):
+        fn(); torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            g.replay()
+        e1.record(); torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / 5
+
     return {
         "split_index_us": timeit(lambda: sg.sg_split_index(hp.shape1, idx, hp.cu_k, Ktot, mask, True, re_, loc, rem, nl, nr)),
         "profile_accumulate_us_per_layer": timeit(lambda: sg.sg_profile_accumulate(hp.shape1, idx, hp.cu_k, Ktot, counts[layer])),
         "block_importance_us": timeit(lambda: sg.sg_block_importance(hp.shape, counts, M, imp)),
         "proactive_mask_us_per_layer": timeit(lambda: sg.sg_proactive_mask(hp.shape1, M, layer, selblk, pmask)),
-        "note": "launch-latency-bound integer kernels (a few KB to a few MB each); eager launches, CUDA events",
+        "push_blocks_us_per_layer": (push_us := timeit_graph(push_all_layers) / L),
+        "push_blocks_gbs": push_bytes / push_us / 1e3,
+        "push_blocks_frac_of_copy_peak": push_bytes / push_us / 1e3 / load_peaks()["hbm_gbs"],
+        "push_blocks_all_layers_one_call_us": (push_all_us := timeit(lambda: sg.sg_push_blocks(hp.shape, M, 0, sel_all, k_cache, v_cache, dst_all_k, dst_all_v))),
+        "push_blocks_all_layers_frac_of_copy_peak": L * push_bytes / push_all_us / 1e3 / load_peaks()["hbm_gbs"],
+        "push_blocks_40pct_one_call_us": (push_40_us := timeit(lambda: sg.sg_push_blocks(hp.shape, M, 0, sel_40, k_cache, v_cache, dst_all_k, dst_all_v))),
+        "push_blocks_40pct_frac_of_copy_peak": 0.4 * L * push_bytes / push_40_us / 1e3 / load_peaks()["hbm_gbs"],
+        "note": "push_blocks moves one whole layer per call (all M = 1024 blocks selected), 32 calls replayed from a CUDA graph; the others are launch-latency-bound integer kernels (a few KB to a few MB each); eager launches, CUDA events",
     }
 
 
@@ -499,7 +531,7 @@ def run_ours(args):
                "score_tflops": work["score"]["flops"] * fr / t["score"] / 1e12}
 
     kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
-    next_rows = next_rows_timing(dev, cfg, hp) if world == 1 else None
+    next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 else None
     sweep = None
     if args.workload == "c2" and not args.no_decode_sweep and world == 1:
         del d_k, d_v, h_k, h_v

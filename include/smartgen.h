@@ -208,6 +208,14 @@ sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const i
  *   available, 2 = on the remote prefill node): tokens whose block's flat id layer*M + m is in `selected`
  *   (int32 [num_selected], ascending -- sg_select_topk's output) get 1, all others 2.  kv_mask int8 [T].
  *   The mask is what sg_split_index consumes.
+ * sg_push_blocks -- the online transfer of one layer (Section 4.1, "Online KV transfer": the layer's cache is
+ *   split into M blocks and every block whose position is among the top-K_r is pushed to the decoding node's
+ *   KV cache pool): for every token of `layer` whose block's flat id layer*M + m is in `selected` (ascending,
+ *   as for sg_proactive_mask), the rows of all KV heads are copied from src_k/src_v to the same positions of
+ *   dst_k/dst_v.  Both caches are bf16, device, addressed with the shape's strides; the call covers the
+ *   shape->num_layers consecutive layers layer, layer + 1, ... (the pointers address the first of them; 1 =
+ *   the paper's layer-by-layer push as each layer is offloaded); rows of other blocks are not written.  The network hop is out of scope: the
+ *   destination is another HBM buffer.  src and dst must not overlap.
  * sg_speculative_delivered -- speculative transfer (Section 4.3; host arithmetic, no GPU): after the prefill
  *   stage pushed the top-K_r blocks, every decoding iteration delivers the next blocks in the order of their
  *   Eq. 1 importance, at most `ratio` of all L*M blocks per iteration (rounded down, at least one).  Returns the
@@ -221,6 +229,9 @@ sg_status sg_block_importance(const sg_shape* shape, const int32_t* counts, int3
 int64_t sg_transfer_budget(int32_t num_layers, int32_t num_blocks, double t_prefill, double t_transfer);
 sg_status sg_proactive_mask(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
                             int32_t num_selected, int8_t* kv_mask, void* stream);
+sg_status sg_push_blocks(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
+                         int32_t num_selected, const void* src_k, const void* src_v, void* dst_k, void* dst_v,
+                         void* stream);
 int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t k_r, double ratio, int32_t iteration);
 
 /*

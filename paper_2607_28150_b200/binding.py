@@ -22,7 +22,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
             "sg_score_static", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
-            "sg_transfer_budget", "sg_proactive_mask", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
+            "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -74,6 +74,8 @@ _lib.sg_speculative_delivered.restype = ctypes.c_int64
 _lib.sg_speculative_delivered.argtypes = [_i32, _i32, ctypes.c_int64, ctypes.c_double, _i32]
 _lib.sg_proactive_mask.restype = ctypes.c_int
 _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
+_lib.sg_push_blocks.restype = ctypes.c_int
+_lib.sg_push_blocks.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_split_index.restype = ctypes.c_int
 _lib.sg_split_index.argtypes = [_sp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn.restype = ctypes.c_int
@@ -266,6 +268,21 @@ def sg_proactive_mask(shape: Shape, num_blocks: int, layer: int, selected: Optio
     rc = _lib.sg_proactive_mask(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(kv_mask), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_proactive_mask")
+
+
+def sg_push_blocks(shape: Shape, num_blocks: int, layer: int, selected: Optional[torch.Tensor], src_k: torch.Tensor,
+                   src_v: torch.Tensor, dst_k: torch.Tensor, dst_v: torch.Tensor, stream=None) -> None:
+    """Online proactive transfer: copy the rows (all KV heads, K and V) of every selected block of the layers
+    `layer` .. `layer + shape.num_layers - 1` from the source cache to the same positions of the destination
+    cache (the tensors start at `layer`); other rows are untouched."""
+    _check(selected, torch.int32, "selected", True)
+    for name, t in (("src_k", src_k), ("src_v", src_v), ("dst_k", dst_k), ("dst_v", dst_v)):
+        _check(t, _BF16, name)
+    n = 0 if selected is None else selected.numel()
+    rc = _lib.sg_push_blocks(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(src_k), _ptr(src_v),
+                             _ptr(dst_k), _ptr(dst_v), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_push_blocks")
 
 
 def sg_speculative_delivered(num_layers: int, num_blocks: int, k_r: int, ratio: float, iteration: int) -> int:
