@@ -268,6 +268,34 @@ def next_rows_timing(dev, cfg, hp, k_cache, v_cache, layer=0, reps=20):
     }
 
 
+def layerwise_prefill_timing(dev, hp, d_q, d_k, d_v, reps=5):
+    """The prefill side issued layer by layer (one score/select/pack call per layer, as a prefill engine would
+    when each layer's KV becomes ready), replayed from a CUDA graph: on one stream, and with select+pack on a
+    second stream so that they overlap the next layer's scoring.  Device ms for all layers."""
+    import torch
+
+    def graph_ms(aux):
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            hp.prefill_layerwise(d_q, d_k, d_v, aux_stream=aux)            # warm-up outside the capture
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                hp.prefill_layerwise(d_q, d_k, d_v, aux_stream=aux)
+            g.replay(); side.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(reps):
+                g.replay()
+            e1.record(side); side.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    one = graph_ms(None)
+    two = graph_ms(torch.cuda.Stream(device=dev))
+    return {"one_stream_ms": one, "two_stream_ms": two, "layers": hp.L,
+            "note": "3 kernels + 1 counter memset per layer; compare with score+select+pack of the all-layer calls in stage_ms"}
+
+
 def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (128, 1.0, 0.5)), calls=16):
     """sg_sparse_decode_attn alone on points of the decode-heavy sweep (B sequences of 4096 tokens, `sel` of the
     prompt required, `rho` of that index-addressed): the sizes at which the kernel can reach the HBM roofline.
@@ -532,6 +560,7 @@ def run_ours(args):
 
     kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
     next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 else None
+    layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 else None
     sweep = None
     if args.workload == "c2" and not args.no_decode_sweep and world == 1:
         del d_k, d_v, h_k, h_v
@@ -553,7 +582,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (3 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "decode_sweep": sweep, "next_rows": next_rows, "dev_status": status, "setup_s": gen_s,
+        "decode_sweep": sweep, "next_rows": next_rows, "prefill_layerwise": layerwise, "dev_status": status, "setup_s": gen_s,
     }
     print(json.dumps(line))
     if world > 1:

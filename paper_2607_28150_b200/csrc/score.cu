@@ -27,6 +27,8 @@
 // work, drains its own TMA copies with bounded waits, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <vector>
+
 #include "common.cuh"
 #include "launch.h"
 
@@ -55,6 +57,7 @@ struct ScoreParams {
   int32_t B, Hkv, G, W, R, Rpad, Ralloc;
   int32_t U;               // units = layers x KV heads
   int32_t lag;             // pass 2 of unit u is scheduled `lag` units after its pass 1
+  int32_t compact;         // schedule layout: 0 = every slot 2*C positions, 1 = positions without an item removed
   int32_t tiles_per_chunk, max_items, k_stages, q_bufs;
   float scale_log2;
 };
@@ -168,6 +171,44 @@ __device__ __forceinline__ uint32_t make_idesc(int M, int N) {
 // with all its sequences (C items per pass).  CTA k walks positions k, k + grid, k + 2*grid, ...  A pass-2
 // item depends only on pass-1 items at smaller positions, and pass-1 items never wait, so the item at the
 // smallest unfinished position can always run: the schedule cannot deadlock whatever the grid size.
+// With few units (lag >= U) the schedule is simply all pass-1 items followed by all pass-2 items.
+struct SchedPos { int pass, unit, j; };    // pass 0 = no item at this position
+__host__ __device__ __forceinline__ long long schedule_length(int U, int C, int lag, bool compact) {
+  return (lag >= U || compact) ? (long long)U * 2 * C : (long long)(U + lag) * 2 * C;
+}
+// Three layouts.  lag >= U (few units): all pass-1 items, then all pass-2 items.  Padded: every slot has
+// 2*C positions, those of units that do not exist are empty (the first and the last `lag` slots are half
+// empty).  Compact: the same order with the empty positions removed.  Which of the last two finishes first
+// depends on how the items fall on the CTAs; the host simulates both and picks (see choose_layout).
+__host__ __device__ __forceinline__ SchedPos schedule_position(long long pos, int U, int C, int lag, bool compact) {
+  SchedPos sp;
+  if (lag >= U) {
+    const long long half = (long long)U * C;
+    const long long q = pos < half ? pos : pos - half;
+    sp.unit = (int)(q / C); sp.j = (int)(q - (long long)sp.unit * C); sp.pass = pos < half ? 1 : 2;
+    return sp;
+  }
+  if (compact) {
+    const long long head = (long long)lag * C, mid = (long long)(U - lag) * 2 * C;
+    if (pos < head) {
+      sp.unit = (int)(pos / C); sp.j = (int)(pos - (long long)sp.unit * C); sp.pass = 1;
+      return sp;
+    }
+    if (pos >= head + mid) {
+      const long long q = pos - head - mid;
+      const int k = (int)(q / C);
+      sp.unit = U - lag + k; sp.j = (int)(q - (long long)k * C); sp.pass = 2;
+      return sp;
+    }
+    pos += head;                                   // inside the middle part both layouts agree up to this shift
+  }
+  const int slot = (int)(pos / (2 * C));
+  const int r = (int)(pos - (long long)slot * (2 * C));
+  if (r < C) { sp.unit = slot - lag; sp.j = r; sp.pass = 2; } else { sp.unit = slot; sp.j = r - C; sp.pass = 1; }
+  if (sp.unit < 0 || sp.unit >= U) sp.pass = 0;
+  return sp;
+}
+
 struct ScoreItem {
   int pass;          // 1 or 2; 0 = no item at this position
   int unit, l, g, b;
@@ -183,11 +224,10 @@ __device__ __forceinline__ ScoreItem decode_position(const ScoreParams& p, long 
   ScoreItem it;
   it.pass = 0;
   const int C = s_prefix[p.B];
-  const int slot = (int)(pos / (2 * C));
-  const int r = (int)(pos - (long long)slot * (2 * C));
-  int unit, j;
-  if (r < C) { unit = slot - p.lag; j = r; it.pass = 2; } else { unit = slot; j = r - C; it.pass = 1; }
-  if (unit < 0 || unit >= p.U) { it.pass = 0; return it; }
+  const SchedPos sp = schedule_position(pos, p.U, C, p.lag, p.compact != 0);
+  it.pass = sp.pass;
+  const int unit = sp.unit, j = sp.j;
+  if (it.pass == 0) return it;
   it.unit = unit;
   it.l = unit / p.Hkv;
   it.g = unit - it.l * p.Hkv;
@@ -296,7 +336,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int C = s_prefix[p.B];
-  const long long npos = (long long)(p.U + p.lag) * 2 * C;
+  const long long npos = schedule_length(p.U, C, p.lag, p.compact != 0);
   volatile int never = 0;
 
   if (warp == 0) {
@@ -674,11 +714,43 @@ ScorePlan plan_score(const sg_shape* s) {
   // still in L2 for the second read.
   const int64_t c_est = (tiles_per_unit - s->batch) / tpc + 1;
   int64_t lag = (5 * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
-  if (lag > pl.U) lag = pl.U;
+  if (2 * lag > pl.U) lag = pl.U;     // few units: all pass-1 items first, then all pass-2 items
   pl.lag = (int)lag;
   pl.counter_bytes = ((size_t)pl.U * sizeof(int) + 255) & ~(size_t)255;
   pl.workspace_bytes = pl.counter_bytes + (size_t)2 * pl.U * pl.max_items * pl.Ralloc * sizeof(float);
   return pl;
+}
+
+// Finish time of the static schedule under a simple model (an item costs its tiles, pass 2 a little more;
+// a pass-2 item starts when its CTA is free and every pass-1 item of its unit is done).  CTA k takes
+// positions k, k + grid, ...; with items of 4-32 tiles, where the empty positions fall decides whether some
+// CTA ends up one item behind, so the host plays both layouts through and keeps the faster.
+double simulate_schedule(int U, int C, int lag, bool compact, int grid, int tiles) {
+  std::vector<double> clock((size_t)grid, 0.0), done1((size_t)U, 0.0);
+  const long long npos = schedule_length(U, C, lag, compact);
+  double end = 0.0;
+  for (long long pos = 0; pos < npos; ++pos) {
+    const SchedPos sp = schedule_position(pos, U, C, lag, compact);
+    if (sp.pass == 0) continue;
+    double& c = clock[(size_t)(pos % grid)];
+    double start = c;
+    if (sp.pass == 2 && done1[(size_t)sp.unit] > start) start = done1[(size_t)sp.unit];
+    c = start + (sp.pass == 2 ? 1.1 : 1.0) * tiles + 1.0;
+    if (sp.pass == 1 && c > done1[(size_t)sp.unit]) done1[(size_t)sp.unit] = c;
+    if (c > end) end = c;
+  }
+  return end;
+}
+
+bool choose_compact_layout(const sg_shape* s, const ScorePlan& pl, int grid) {
+  if (pl.lag >= pl.U) return false;                               // two-phase schedule: nothing to choose
+  // items per unit and pass: exact for one sequence, an estimate for a ragged batch (lengths live on the device)
+  const long long tiles_per_unit = s->batch == 1 ? ((long long)s->total_tokens + kTileKeys - 1) / kTileKeys
+                                                 : (long long)s->total_tokens / kTileKeys + (s->batch + 1) / 2;
+  const int C = (int)((tiles_per_unit + pl.tiles_per_chunk - 1) / pl.tiles_per_chunk);
+  if (schedule_length(pl.U, C, pl.lag, false) > 40000) return false;   // long schedules: the ends do not matter
+  return simulate_schedule(pl.U, C, pl.lag, true, grid, pl.tiles_per_chunk) <
+         simulate_schedule(pl.U, C, pl.lag, false, grid, pl.tiles_per_chunk);
 }
 
 }  // namespace
@@ -769,6 +841,7 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = kNumSMs;
   const long long max_pos = (long long)(pl.U + pl.lag) * 2 * pl.max_items;
   const unsigned grid = (unsigned)(max_pos < sms ? max_pos : sms);     // persistent: one CTA per SM
+  p.compact = choose_compact_layout(shape, pl, (int)grid) ? 1 : 0;
   if (D == 128) {
     SG_ENSURE_SMEM((score_kernel<128>), pl.smem_bytes);
     score_kernel<128><<<grid, kScoreThreads, pl.smem_bytes, s>>>(tmap_q, tmap_k, p);

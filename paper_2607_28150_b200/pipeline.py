@@ -3,7 +3,8 @@
 `HotPath` owns the device buffers of one batch of prompts -- importance, KV index, packed K/V,
 workspaces, status word -- and issues the library calls in the order of the path:
 
-    prefill side:  sg_score -> sg_select_topk -> sg_pack_kv      (all layers in one call each)
+    prefill side:  sg_score -> sg_select_topk -> sg_pack_kv      (all layers in one call each, or layer by
+                                                                   layer with select+pack on a second stream)
     decode side :  sg_sparse_decode_attn                          (one call per layer per step)
 
 No arithmetic of the method happens here; every step runs in the library's CUDA kernels.
@@ -70,6 +71,40 @@ class HotPath:
         self.score(q_win, k_cache, stream)
         self.select(stream)
         return self.pack(k_cache, v_cache, stream)
+
+    def prefill_layer(self, layer: int, q_win: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                      stream=None, aux_stream=None):
+        """score -> select -> pack of ONE layer, as a prefill engine calls them when that layer's KV is ready
+        (the paper transfers layer by layer, overlapped with the prefill of the following layers).
+        `q_win`, `k_cache`, `v_cache` are the full [L][...] tensors.  With `aux_stream`, select and pack run
+        there behind an event, so the next layer's scoring on `stream` does not wait for them; the caller joins
+        with `join_aux` before reading the results on `stream`."""
+        main = stream if stream is not None else torch.cuda.current_stream(self.device)
+        sg.sg_score(self.shape1, q_win[layer], k_cache[layer], self.importance[layer], self.ws_score, self.status, main)
+        side = main
+        if aux_stream is not None:
+            ev = torch.cuda.Event()
+            ev.record(main)
+            aux_stream.wait_event(ev)
+            side = aux_stream
+        sg.sg_select_topk(self.shape1, self.importance[layer], self.cu_k, self.K_tot, self.sel_idx[layer], None,
+                          self.status, side)
+        sg.sg_pack_kv(self.shape1, k_cache[layer], v_cache[layer], self.sel_idx[layer], self.cu_k, self.K_tot,
+                      self.packed_k[layer], self.packed_v[layer], self.status, side)
+
+    def join_aux(self, aux_stream, stream=None) -> None:
+        """Make `stream` wait for everything queued on `aux_stream` so far."""
+        main = stream if stream is not None else torch.cuda.current_stream(self.device)
+        ev = torch.cuda.Event()
+        ev.record(aux_stream)
+        main.wait_event(ev)
+
+    def prefill_layerwise(self, q_win, k_cache, v_cache, stream=None, aux_stream=None):
+        for layer in range(self.L):
+            self.prefill_layer(layer, q_win, k_cache, v_cache, stream, aux_stream)
+        if aux_stream is not None:
+            self.join_aux(aux_stream, stream)
+        return self.packed_k, self.packed_v
 
     # ---- decode side --------------------------------------------------------------------------
     def decode_workspace(self, total_loc: int) -> torch.Tensor:

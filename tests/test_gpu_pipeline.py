@@ -63,3 +63,28 @@ def test_tiny_config_end_to_end_decode():
     got_o, got_l = gpu_ops.sparse_decode_attn(q, pk[0], pv[0], ck, data["k"][0], data["v"][0], cu, loc, cl)
     want_o, want_l = oracle.sparse_decode_attn(q, pk[0], pv[0], ck, data["k"][0], data["v"][0], cu, loc, cl)
     assert np.abs(got_o - want_o).max() <= 2e-2 and np.abs(got_l - want_l).max() <= 1e-3
+
+
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_layer_by_layer_prefill_matches_the_oracle_chain(two_streams):
+    """score -> select -> pack issued layer by layer (optionally with select+pack on a second stream): scores within
+    tolerance of the oracle, and index sets / packed bytes bit-exact against the oracle run on those same scores."""
+    import torch
+    from paper_2607_28150_b200.pipeline import HotPath, as_device
+    cfg = wl.varlen(0.1, seqlens=(1500, 4096, 130), num_layers=5)
+    data = wl.make_prefill(cfg)
+    cu, ck = data["cu_seqlens"], cfg.cu_k()
+    hp = HotPath(cfg.num_layers, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.window, cfg.seqlens, cfg.budgets())
+    q, k, v = as_device(data["q_win"]), as_device(data["k"]), as_device(data["v"])
+    aux = torch.cuda.Stream() if two_streams else None
+    hp.prefill_layerwise(q, k, v, aux_stream=aux)
+    torch.cuda.synchronize()
+    assert hp.read_status() == 0
+    imp_g = hp.importance.cpu().numpy()
+    imp_o = oracle.score(data["q_win"], data["k"], cu)
+    assert np.all(np.abs(imp_g - imp_o) <= 1e-4 * np.abs(imp_o) + 1e-30)
+    sel_o = oracle.select_topk(imp_g, cu, ck)
+    assert np.array_equal(hp.sel_idx.cpu().numpy(), sel_o)
+    pk_o, pv_o = oracle.pack_kv(data["k"], data["v"], cu, sel_o, ck)
+    assert np.array_equal(hp.packed_k.cpu().numpy().view(np.uint16), pk_o)
+    assert np.array_equal(hp.packed_v.cpu().numpy().view(np.uint16), pv_o)
