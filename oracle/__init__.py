@@ -87,6 +87,22 @@ def select_topk(importance: np.ndarray, cu_seqlens: np.ndarray, cu_k: np.ndarray
     return sel
 
 
+def select_threshold(scores: np.ndarray, cu_seqlens: np.ndarray, alpha: float, cu_cap: np.ndarray):
+    """Threshold selection: per (layer, sequence, KV head) the tokens with score > row max - alpha, at most
+    cap_b of them (the largest, ties to the lower index).  Returns sel_idx int32 [L][H_kv][cap_tot] (ascending,
+    then -1) and sel_count int32 [L][B][H_kv]."""
+    x, cu, cc = _c(scores, np.float32), _c(cu_seqlens, np.int32), _c(cu_cap, np.int32)
+    L, Hkv, T = x.shape
+    B = cu.shape[0] - 1
+    assert cu[-1] == T and cc.shape == (B + 1,)
+    sel = np.zeros((L, Hkv, int(cc[-1])), dtype=np.int32)
+    cnt = np.zeros((L, B, Hkv), dtype=np.int32)
+    rc = _load().sgo_select_threshold(L, B, Hkv, _p(cu), _p(x), ctypes.c_float(alpha), _p(cc), _p(sel), _p(cnt))
+    if rc:
+        raise RuntimeError("sgo_select_threshold failed: %d" % rc)
+    return sel, cnt
+
+
 def pack_kv(k_cache: np.ndarray, v_cache: np.ndarray, cu_seqlens: np.ndarray, sel_idx: np.ndarray, cu_k: np.ndarray):
     """packed_k, packed_v uint16 [L][K_tot*H_kv][d]; row of (b, g, j) is cu_k[b]*H_kv + g*k_b + j."""
     k, v = _c(k_cache, np.uint16), _c(v_cache, np.uint16)

@@ -440,3 +440,47 @@ int sgo_push_blocks(int B, int Hkv, int d, int M, const int32_t *cu, int layer, 
     }
     return 0;
 }
+
+/* Threshold selection (the selection rule of the KV selection algorithm the paper deploys, Section 5.1
+ * "Parameters": an alpha value and a maximum KV selection ratio): per (layer, sequence, KV head) every token
+ * whose score exceeds the row maximum minus alpha is selected, at most cap_b = cu_cap[b+1] - cu_cap[b] of them;
+ * if more exceed the threshold, the cap_b largest are kept (ties to the lower index).
+ * scores float [L][Hkv][T]; sel_idx int32 [L][Hkv][cap_tot]: the selected positions in ascending order, then -1;
+ * sel_count int32 [L][B][Hkv].  NaN scores are never selected.  Returns 2 for a cap outside [0, N_b]. */
+int sgo_select_threshold(int L, int B, int Hkv, const int32_t *cu, const float *scores, float alpha,
+                         const int32_t *cu_cap, int32_t *sel_idx, int32_t *sel_count) {
+    const int64_t T = cu[B], cap_tot = cu_cap[B];
+    for (int b = 0; b < B; ++b) {
+        const int cap = cu_cap[b + 1] - cu_cap[b];
+        if (cap < 0 || cap > cu[b + 1] - cu[b]) return 2;
+    }
+    for (int l = 0; l < L; ++l)
+        for (int b = 0; b < B; ++b)
+            for (int g = 0; g < Hkv; ++g) {
+                const int N = cu[b + 1] - cu[b];
+                const int cap = cu_cap[b + 1] - cu_cap[b];
+                const float *x = scores + ((int64_t)l * Hkv + g) * T + cu[b];
+                int32_t *out = sel_idx + ((int64_t)l * Hkv + g) * cap_tot + cu_cap[b];
+                int have_max = 0;
+                float m = 0.0f;
+                for (int t = 0; t < N; ++t)
+                    if (x[t] == x[t] && (!have_max || x[t] > m)) { m = x[t]; have_max = 1; }
+                const float thr = m - alpha;                         /* single precision, as the scores are */
+                sgo_pair *p = (sgo_pair *)malloc((size_t)(N > 0 ? N : 1) * sizeof(sgo_pair));
+                if (!p) return 1;
+                int n = 0;
+                if (have_max)
+                    for (int t = 0; t < N; ++t)
+                        if (x[t] > thr) { p[n].key = order_key(x[t]); p[n].t = t; ++n; }
+                if (n > cap) {
+                    qsort(p, (size_t)n, sizeof(sgo_pair), cmp_key_desc_index_asc);
+                    n = cap;
+                }
+                for (int j = 0; j < n; ++j) out[j] = p[j].t;
+                qsort(out, (size_t)n, sizeof(int32_t), cmp_int_asc);
+                for (int j = n; j < cap; ++j) out[j] = -1;
+                sel_count[((int64_t)l * B + b) * Hkv + g] = n;
+                free(p);
+            }
+    return 0;
+}
