@@ -226,6 +226,12 @@ def next_rows_timing(dev, cfg, hp, k_cache, v_cache, layer=0, reps=20):
         for l in range(L):
             sg.sg_push_blocks(hp.shape1, M, l, push_sel[l], k_cache[l], v_cache[l], dst_k, dst_v)
     push_bytes = 2 * 2 * T * Hkv * hp.d * 2
+    # threshold selection on the step's importance: alpha = 2 of the R = G*W attention mass, cap 20 % of each prompt
+    caps = [max(1, -(-int(n) // 5)) for n in np.diff(hp.cu_host)]
+    cu_cap = torch.tensor(np.concatenate([[0], np.cumsum(caps)]).astype(np.int32), device=dev)
+    cap_tot = int(sum(caps))
+    thr_idx = torch.empty((L, Hkv, cap_tot), dtype=torch.int32, device=dev)
+    thr_cnt = torch.empty((L, B, Hkv), dtype=torch.int32, device=dev)
     dst_all_k = torch.empty_like(k_cache); dst_all_v = torch.empty_like(v_cache)
     sel_all = torch.arange(0, L * M, dtype=torch.int32, device=dev)
     sel_40 = torch.arange(0, L * M, dtype=torch.int32, device=dev)[torch.randperm(L * M, generator=gen, device=dev)[: (2 * L * M) // 5]].sort().values.contiguous()
@@ -257,6 +263,7 @@ def next_rows_timing(dev, cfg, hp, k_cache, v_cache, layer=0, reps=20):
         "profile_accumulate_us_per_layer": timeit(lambda: sg.sg_profile_accumulate(hp.shape1, idx, hp.cu_k, Ktot, counts[layer])),
         "block_importance_us": timeit(lambda: sg.sg_block_importance(hp.shape, counts, M, imp)),
         "proactive_mask_us_per_layer": timeit(lambda: sg.sg_proactive_mask(hp.shape1, M, layer, selblk, pmask)),
+        "select_threshold_all_layers_us": timeit(lambda: sg.sg_select_threshold(hp.shape, hp.importance, 2.0, cu_cap, cap_tot, thr_idx, thr_cnt)),
         "push_blocks_us_per_layer": (push_us := timeit_graph(push_all_layers) / L),
         "push_blocks_gbs": push_bytes / push_us / 1e3,
         "push_blocks_frac_of_copy_peak": push_bytes / push_us / 1e3 / load_peaks()["hbm_gbs"],

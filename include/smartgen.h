@@ -235,6 +235,26 @@ sg_status sg_push_blocks(const sg_shape* shape, int32_t num_blocks, int32_t laye
 int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t k_r, double ratio, int32_t iteration);
 
 /*
+ * sg_select_threshold -- threshold selection under a cap, the rule of the KV selection algorithm the paper
+ * deploys (Section 5.1, "Parameters": an alpha value and a maximum KV selection ratio): per (layer, sequence,
+ * KV head) every token whose score exceeds the row maximum minus `alpha` is selected, at most
+ * cap_b = cu_cap[b+1] - cu_cap[b] of them; if more exceed the threshold the cap_b largest are kept, ties to the
+ * lower index.  The comparison is strict.  Scores must not be NaN (sg_score never produces one): a NaN is never
+ * selected, but which of the other tokens of its row are is then unspecified (always in range, never a fault).
+ *   scores    fp32 [L][H_kv][T], device (any per-token score; sg_score's importance has this layout)
+ *   alpha     >= 0, in the units of the scores
+ *   cu_cap    int32 [B+1], device: prefix sums of the caps (0 <= cap_b <= N_b), total_cap = cu_cap[B] on the host
+ *   sel_idx   int32 [L][H_kv][total_cap], device, written: per row the selected sequence-local positions in
+ *             ascending order, then -1 up to cap_b
+ *   sel_count int32 [L][B][H_kv], device, written: the number selected per row
+ * Runs sg_select_topk with the caps as budgets, then trims each row at the threshold; the counts differ per KV
+ * head, so the rows are not directly consumable by sg_pack_kv (which takes one budget per sequence).
+ * Errors as sg_select_topk.
+ */
+sg_status sg_select_threshold(const sg_shape* shape, const float* scores, float alpha, const int32_t* cu_cap,
+                              int32_t total_cap, int32_t* sel_idx, int32_t* sel_count, int32_t* dev_status, void* stream);
+
+/*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.
  *
  * The paper has no counterpart to this call: it computes exactly what sg_score computes.  It exists

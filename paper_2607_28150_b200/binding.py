@@ -21,7 +21,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_score_static", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
+            "sg_score_static", "sg_select_threshold", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
             "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -74,6 +74,8 @@ _lib.sg_speculative_delivered.restype = ctypes.c_int64
 _lib.sg_speculative_delivered.argtypes = [_i32, _i32, ctypes.c_int64, ctypes.c_double, _i32]
 _lib.sg_proactive_mask.restype = ctypes.c_int
 _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
+_lib.sg_select_threshold.restype = ctypes.c_int
+_lib.sg_select_threshold.argtypes = [_sp, _vp, _f, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.sg_push_blocks.restype = ctypes.c_int
 _lib.sg_push_blocks.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_split_index.restype = ctypes.c_int
@@ -268,6 +270,20 @@ def sg_proactive_mask(shape: Shape, num_blocks: int, layer: int, selected: Optio
     rc = _lib.sg_proactive_mask(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(kv_mask), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_proactive_mask")
+
+
+def sg_select_threshold(shape: Shape, scores: torch.Tensor, alpha: float, cu_cap: torch.Tensor, total_cap: int,
+                        sel_idx: torch.Tensor, sel_count: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                        stream=None) -> None:
+    """Threshold selection under a cap: per row the positions with score > row max - alpha (at most cap_b, the
+    largest first, ties to the lower index), ascending then -1, plus the count per (layer, sequence, KV head)."""
+    _check(scores, torch.float32, "scores"); _check(cu_cap, torch.int32, "cu_cap")
+    _check(sel_idx, torch.int32, "sel_idx", total_cap == 0); _check(sel_count, torch.int32, "sel_count")
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_select_threshold(ctypes.byref(shape), _ptr(scores), alpha, _ptr(cu_cap), total_cap, _ptr(sel_idx),
+                                  _ptr(sel_count), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_select_threshold")
 
 
 def sg_push_blocks(shape: Shape, num_blocks: int, layer: int, selected: Optional[torch.Tensor], src_k: torch.Tensor,
