@@ -103,29 +103,35 @@ def select_threshold(scores: np.ndarray, cu_seqlens: np.ndarray, alpha: float, c
     return sel, cnt
 
 
-def pack_kv(k_cache: np.ndarray, v_cache: np.ndarray, cu_seqlens: np.ndarray, sel_idx: np.ndarray, cu_k: np.ndarray):
-    """packed_k, packed_v uint16 [L][K_tot*H_kv][d]; row of (b, g, j) is cu_k[b]*H_kv + g*k_b + j."""
+def pack_kv(k_cache: np.ndarray, v_cache: np.ndarray, cu_seqlens: np.ndarray, sel_idx: np.ndarray, cu_k: np.ndarray,
+            sel_count: Optional[np.ndarray] = None, fill: int = 0):
+    """packed_k, packed_v uint16 [L][K_tot*H_kv][d]; row of (b, g, j) is cu_k[b]*H_kv + g*k_b + j.
+    With sel_count (int32 [L][B][H_kv]) only the first sel_count[l][b][g] entries of each row are packed; the other
+    rows keep `fill`."""
     k, v = _c(k_cache, np.uint16), _c(v_cache, np.uint16)
     cu, ck, sel = _c(cu_seqlens, np.int32), _c(cu_k, np.int32), _c(sel_idx, np.int32)
     L, T, Hkv, d = k.shape
     B = cu.shape[0] - 1
     Ktot = int(ck[-1])
     assert v.shape == k.shape and sel.shape == (L, Hkv, Ktot)
-    pk = np.zeros((L, Ktot * Hkv, d), dtype=np.uint16)
-    pv = np.zeros_like(pk)
+    pk = np.full((L, Ktot * Hkv, d), fill, dtype=np.uint16)
+    pv = np.full_like(pk, fill)
+    sc = None if sel_count is None else _c(sel_count, np.int32)
+    assert sc is None or sc.shape == (L, B, Hkv)
     rc = _load().sgo_pack_kv(L, B, Hkv, d, _p(cu), _p(k), _p(v), _i64(T * Hkv * d), _i64(Hkv * d), _i64(d),
-                             _p(sel), _p(ck), _p(pk), _p(pv))
+                             _p(sel), _p(ck), _p(pk), _p(pv), None if sc is None else _p(sc))
     if rc:
         raise RuntimeError("sgo_pack_kv failed: %d" % rc)
     return pk, pv
 
 
 def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu_seqlens, local_idx, cu_nloc,
-                       softmax_scale: float = 0.0):
+                       softmax_scale: float = 0.0, packed_count: Optional[np.ndarray] = None):
     """(out float32 [B][H_q][d], lse float32 [B][H_q]) of attention over packed rows ++ indexed local rows.
 
     q uint16 [B][H_q][d]; packed_k/v uint16 [K_tot*H_kv][d]; local_k/v uint16 [T][H_kv][d];
-    local_idx int32 [H_kv][NL_tot].
+    local_idx int32 [H_kv][NL_tot].  With packed_count (int32 [B][H_kv]) only the first packed_count[b][g] packed rows
+    of each (sequence, KV head) are attended.
     """
     q, pk, pv = _c(q, np.uint16), _c(packed_k, np.uint16), _c(packed_v, np.uint16)
     lk, lv = _c(local_k, np.uint16), _c(local_v, np.uint16)
@@ -137,7 +143,7 @@ def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu_seqlens
     lse = np.zeros((B, Hq), dtype=np.float32)
     rc = _load().sgo_sparse_decode_attn(B, Hq, Hkv, d, _p(cu), _p(q), _p(pk), _p(pv), _p(ck), _p(lk), _p(lv),
                                         _i64(Hkv * d), _i64(d), _p(li), _p(cl), ctypes.c_double(softmax_scale),
-                                        _p(out), _p(lse))
+                                        _p(out), _p(lse), None if packed_count is None else _p(_c(packed_count, np.int32)))
     if rc:
         raise RuntimeError("sgo_sparse_decode_attn failed: %d" % rc)
     return out, lse

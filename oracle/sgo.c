@@ -174,7 +174,9 @@ int sgo_select_topk(int L, int B, int Hkv, const int32_t *cu, const float *impor
  */
 int sgo_pack_kv(int L, int B, int Hkv, int d, const int32_t *cu, const uint16_t *k_cache,
                 const uint16_t *v_cache, int64_t ls, int64_t ts, int64_t hs, const int32_t *sel_idx,
-                const int32_t *cu_k, uint16_t *packed_k, uint16_t *packed_v) {
+                const int32_t *cu_k, uint16_t *packed_k, uint16_t *packed_v, const int32_t *sel_count) {
+    /* sel_count (int32 [L][B][Hkv], may be NULL): only the first sel_count[l][b][g] entries of a row of the KV index
+     * are selected (threshold selection); the remaining rows of the head's slot in the buffer are left as they are. */
     const int64_t K_tot = cu_k[B];
     int bad = 0;
     for (int l = 0; l < L; ++l)
@@ -182,7 +184,13 @@ int sgo_pack_kv(int L, int B, int Hkv, int d, const int32_t *cu, const uint16_t 
             for (int g = 0; g < Hkv; ++g) {
                 const int N = cu[b + 1] - cu[b];
                 const int kb = cu_k[b + 1] - cu_k[b];
-                for (int j = 0; j < kb; ++j) {
+                int kbe = kb;
+                if (sel_count) {
+                    kbe = sel_count[((int64_t)l * B + b) * Hkv + g];
+                    if (kbe < 0) kbe = 0;
+                    if (kbe > kb) kbe = kb;
+                }
+                for (int j = 0; j < kbe; ++j) {
                     const int32_t t = sel_idx[((int64_t)l * Hkv + g) * K_tot + cu_k[b] + j];
                     if (t < 0 || t >= N) { bad = 3; continue; }
                     const int64_t src = l * ls + ((int64_t)cu[b] + t) * ts + g * hs;
@@ -207,12 +215,14 @@ int sgo_pack_kv(int L, int B, int Hkv, int d, const int32_t *cu, const uint16_t 
  * local_k/v bf16, element (token, g, c) at token*ts + g*hs + c; local_idx int32 [Hkv][NL_tot].
  * out float [B][Hq][d] (not rounded to bf16); lse float [B][Hq] = max + ln(sum).
  * An empty list gives out = 0 and lse = -inf.  Returns 3 on an out-of-range local index.
+ * packed_count (int32 [B][Hkv], may be NULL): when the selection kept a different number of entries per KV head
+ * (threshold selection), only the first packed_count[b][g] of the k_b packed rows of (b, g) are in the list.
  */
 int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, const uint16_t *q,
                            const uint16_t *packed_k, const uint16_t *packed_v, const int32_t *cu_k,
                            const uint16_t *local_k, const uint16_t *local_v, int64_t ts, int64_t hs,
                            const int32_t *local_idx, const int32_t *cu_nloc, double softmax_scale,
-                           float *out, float *lse) {
+                           float *out, float *lse, const int32_t *packed_count) {
     if (Hkv <= 0 || Hq % Hkv != 0) return 1;
     const int G = Hq / Hkv;
     const int64_t NL_tot = cu_nloc[B];
@@ -224,8 +234,14 @@ int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, con
             const int g = h / G;
             const int N = cu[b + 1] - cu[b];
             const int kb = cu_k[b + 1] - cu_k[b];
+            int kbe = kb;                                        /* packed rows actually in the list */
+            if (packed_count) {
+                kbe = packed_count[(int64_t)b * Hkv + g];
+                if (kbe < 0) kbe = 0;
+                if (kbe > kb) kbe = kb;
+            }
             const int nl = cu_nloc[b + 1] - cu_nloc[b];
-            const int n = kb + nl;
+            const int n = kbe + nl;
             float *o = out + ((int64_t)b * Hq + h) * d;
             for (int c = 0; c < d; ++c) o[c] = 0.0f;
             if (lse) lse[(int64_t)b * Hq + h] = -INFINITY;
@@ -235,7 +251,7 @@ int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, con
             double *s = (double *)malloc((size_t)n * sizeof(double));
             double *acc = (double *)calloc((size_t)d, sizeof(double));
             int m = 0;
-            for (int j = 0; j < kb; ++j, ++m) {
+            for (int j = 0; j < kbe; ++j, ++m) {
                 const int64_t row = ((int64_t)cu_k[b] * Hkv + (int64_t)g * kb + j) * d;
                 kr[m] = packed_k + row;
                 vr[m] = packed_v + row;

@@ -75,3 +75,40 @@ def test_ties_at_the_cap_go_to_the_lower_index_and_nan_is_never_selected():
     assert cnt[0, 0, 0] == 3 and sel[0, 0].tolist() == [1, 2, 3]
     sel, cnt = oracle.select_threshold(x, cu, 1.0, cu_of((8,)))
     assert sel[0, 0, :cnt[0, 0, 0]].tolist() == [1, 2, 3, 5, 7]
+
+
+def test_counted_pack_and_decode_equal_the_plain_path_on_the_trimmed_selection():
+    """Ragged per-head counts: packing the first count entries of each row and attending only those packed rows is the
+    same as the plain path run head by head with that head's own budget (the definition of the plain path)."""
+    from helpers import rand_bf16
+    rng = np.random.default_rng(5)
+    lens, caps, Hq, Hkv, d = (60, 33), (12, 7), 4, 2, 16
+    cu, cc = cu_of(lens), cu_of(caps)
+    T = int(cu[-1])
+    k, v = rand_bf16(rng, (1, T, Hkv, d)), rand_bf16(rng, (1, T, Hkv, d))
+    q = rand_bf16(rng, (len(lens), Hq, d))
+    x = rng.standard_normal((1, Hkv, T)).astype(np.float32)
+    sel, cnt = oracle.select_threshold(x, cu, 0.8, cc)
+    assert len(set(cnt.ravel().tolist())) > 1                      # counts really differ per head
+    pk, pv = oracle.pack_kv(k, v, cu, sel, cc, sel_count=cnt, fill=0x7fc0)
+    loc = np.zeros((Hkv, 0), dtype=np.int32)
+    out, lse = oracle.sparse_decode_attn(q, pk[0], pv[0], cc, k[0], v[0], cu, loc, cu_of((0, 0)), packed_count=cnt[0])
+    G = Hq // Hkv
+    for g in range(Hkv):                                           # one KV head at a time, uniform budget = that head's count
+        for b in range(len(lens)):
+            n = int(cnt[0, b, g])
+            rows = pk[0].reshape(-1, d)[cc[b] * Hkv + g * caps[b]: cc[b] * Hkv + g * caps[b] + n]
+            want_rows = k[0, cu[b] + sel[0, g, cc[b]:cc[b] + n], g]
+            assert np.array_equal(rows, want_rows)
+            rest = pk[0].reshape(-1, d)[cc[b] * Hkv + g * caps[b] + n: cc[b] * Hkv + (g + 1) * caps[b]]
+            assert np.all(rest == 0x7fc0)                          # rows beyond the count are not written
+            if n == 0:
+                assert np.all(out[b, g * G:(g + 1) * G] == 0) and np.all(np.isneginf(lse[b, g * G:(g + 1) * G]))
+                continue
+            # dense attention over exactly those tokens, in numpy
+            from helpers import widen
+            kk, vv = widen(k[0, cu[b] + sel[0, g, cc[b]:cc[b] + n], g]), widen(v[0, cu[b] + sel[0, g, cc[b]:cc[b] + n], g])
+            for h in range(g * G, (g + 1) * G):
+                s = kk @ widen(q[b, h]) / np.sqrt(d)
+                p = np.exp(s - s.max()); p /= p.sum()
+                assert np.allclose(out[b, h], p @ vv, atol=1e-6)
