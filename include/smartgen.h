@@ -248,11 +248,34 @@ int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t
  *             ascending order, then -1 up to cap_b
  *   sel_count int32 [L][B][H_kv], device, written: the number selected per row
  * Runs sg_select_topk with the caps as budgets, then trims each row at the threshold; the counts differ per KV
- * head, so the rows are not directly consumable by sg_pack_kv (which takes one budget per sequence).
+ * head, so the rows go to sg_pack_kv_counted / sg_sparse_decode_attn_counted (sg_pack_kv takes one budget per
+ * sequence).
  * Errors as sg_select_topk.
  */
 sg_status sg_select_threshold(const sg_shape* shape, const float* scores, float alpha, const int32_t* cu_cap,
                               int32_t total_cap, int32_t* sel_idx, int32_t* sel_count, int32_t* dev_status, void* stream);
+
+/*
+ * sg_pack_kv_counted, sg_sparse_decode_attn_counted -- the gather-pack and the decode attention for a selection
+ * that kept a different number of entries per KV head (sg_select_threshold).  The packed buffer keeps the layout
+ * of sg_pack_kv with the caps as budgets (row of (b, g, j) = cu_cap[b]*H_kv + g*cap_b + j), so every head owns a
+ * slot of cap_b rows, of which only the first count are meaningful:
+ *   sg_pack_kv_counted            sel_count int32 [L][B][H_kv], device: entries j >= sel_count[l][b][g] of a row of
+ *                                 sel_idx are skipped (not read, their rows of packed_k/packed_v not written);
+ *                                 everything else as sg_pack_kv with cu_cap / total_cap in place of cu_k / total_sel.
+ *   sg_sparse_decode_attn_counted packed_count int32 [B][H_kv], device (one layer's slice of sel_count): the list of
+ *                                 (b, g) is its first packed_count[b][g] packed rows, then its local rows; values
+ *                                 are clamped to [0, cap_b].  No workspace.  Everything else as sg_sparse_decode_attn.
+ * With every count equal to its cap the two calls are sg_pack_kv and sg_sparse_decode_attn.
+ */
+sg_status sg_pack_kv_counted(const sg_shape* shape, const void* k_cache, const void* v_cache, const int32_t* sel_idx,
+                             const int32_t* cu_cap, int32_t total_cap, const int32_t* sel_count, void* packed_k,
+                             void* packed_v, int32_t* dev_status, void* stream);
+sg_status sg_sparse_decode_attn_counted(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v,
+                                        const int32_t* cu_cap, int32_t total_cap, const int32_t* packed_count,
+                                        const void* local_k, const void* local_v, const int32_t* local_idx,
+                                        const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
+                                        float* lse, int32_t* dev_status, void* stream);
 
 /*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.

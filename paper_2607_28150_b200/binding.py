@@ -21,7 +21,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_score_static", "sg_select_threshold", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
+            "sg_score_static", "sg_select_threshold", "sg_pack_kv_counted", "sg_sparse_decode_attn_counted", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
             "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -74,6 +74,10 @@ _lib.sg_speculative_delivered.restype = ctypes.c_int64
 _lib.sg_speculative_delivered.argtypes = [_i32, _i32, ctypes.c_int64, ctypes.c_double, _i32]
 _lib.sg_proactive_mask.restype = ctypes.c_int
 _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
+_lib.sg_pack_kv_counted.restype = ctypes.c_int
+_lib.sg_pack_kv_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_sparse_decode_attn_counted.restype = ctypes.c_int
+_lib.sg_sparse_decode_attn_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp, _vp]
 _lib.sg_select_threshold.restype = ctypes.c_int
 _lib.sg_select_threshold.argtypes = [_sp, _vp, _f, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.sg_push_blocks.restype = ctypes.c_int
@@ -284,6 +288,41 @@ def sg_select_threshold(shape: Shape, scores: torch.Tensor, alpha: float, cu_cap
                                   _ptr(sel_count), _ptr(dev_status), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_select_threshold")
+
+
+def sg_pack_kv_counted(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tensor, sel_idx: torch.Tensor,
+                       cu_cap: torch.Tensor, total_cap: int, sel_count: torch.Tensor, packed_k: torch.Tensor,
+                       packed_v: torch.Tensor, dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """sg_pack_kv for per-head counts: only the first sel_count[l][b][g] entries of each row of sel_idx are packed."""
+    _check(k_cache, _BF16, "k_cache"); _check(v_cache, _BF16, "v_cache"); _check(sel_idx, torch.int32, "sel_idx", total_cap == 0)
+    _check(cu_cap, torch.int32, "cu_cap"); _check(sel_count, torch.int32, "sel_count")
+    _check(packed_k, _BF16, "packed_k", total_cap == 0); _check(packed_v, _BF16, "packed_v", total_cap == 0)
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_pack_kv_counted(ctypes.byref(shape), _ptr(k_cache), _ptr(v_cache), _ptr(sel_idx), _ptr(cu_cap), total_cap,
+                                 _ptr(sel_count), _ptr(packed_k), _ptr(packed_v), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_pack_kv_counted")
+
+
+def sg_sparse_decode_attn_counted(shape: Shape, q: torch.Tensor, packed_k: Optional[torch.Tensor], packed_v: Optional[torch.Tensor],
+                                  cu_cap: torch.Tensor, total_cap: int, packed_count: torch.Tensor,
+                                  local_k: Optional[torch.Tensor], local_v: Optional[torch.Tensor],
+                                  local_idx: Optional[torch.Tensor], cu_nloc: torch.Tensor, total_loc: int, out: torch.Tensor,
+                                  lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                                  dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """sg_sparse_decode_attn for per-head counts: of the cap_b packed rows of (b, g) only the first packed_count[b][g]
+    are attended."""
+    _check(q, _BF16, "q"); _check(out, _BF16, "out"); _check(cu_cap, torch.int32, "cu_cap"); _check(cu_nloc, torch.int32, "cu_nloc")
+    _check(packed_count, torch.int32, "packed_count")
+    _check(packed_k, _BF16, "packed_k", True); _check(packed_v, _BF16, "packed_v", True)
+    _check(local_k, _BF16, "local_k", True); _check(local_v, _BF16, "local_v", True)
+    _check(local_idx, torch.int32, "local_idx", True); _check(lse, torch.float32, "lse", True)
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_sparse_decode_attn_counted(ctypes.byref(shape), _ptr(q), _ptr(packed_k), _ptr(packed_v), _ptr(cu_cap), total_cap,
+                                            _ptr(packed_count), _ptr(local_k), _ptr(local_v), _ptr(local_idx), _ptr(cu_nloc),
+                                            total_loc, softmax_scale, _ptr(out), _ptr(lse), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_sparse_decode_attn_counted")
 
 
 def sg_push_blocks(shape: Shape, num_blocks: int, layer: int, selected: Optional[torch.Tensor], src_k: torch.Tensor,

@@ -40,6 +40,7 @@ struct DecParams {
   const int32_t* cu_k;
   const int32_t* cu_nloc;
   const int32_t* local_idx;
+  const int32_t* packed_count;   // [B][Hkv] packed rows of a (sequence, KV head) that are in the list, or null: all k_b
   uint16_t* out;
   float* lse;
   int32_t* dev_status;
@@ -118,14 +119,15 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   if (p.csize > 1) cluster_arrive_relaxed();                   // "this CTA runs": awaited before the first remote store
   const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
-  const int kb = p.cu_k[b + 1] - p.cu_k[b];
+  const int kb = p.cu_k[b + 1] - p.cu_k[b];                    // packed rows per KV head (the slot size in the buffer)
+  const int kbe = p.packed_count ? min(kb, max(0, __ldg(p.packed_count + (int64_t)b * p.Hkv + g))) : kb;   // ... of which in the list
   const int nl = p.cu_nloc[b + 1] - p.cu_nloc[b];
   const int c0 = p.cu[b];
   const int nseq = p.cu[b + 1] - c0;
   // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
-  const int span = ((((kb + nl + p.csize - 1) / p.csize) + kSlice - 1) / kSlice) * kSlice;
-  const int range_beg = min(kb + nl, c * span);
-  const int range_end = min(kb + nl, range_beg + span);
+  const int span = ((((kbe + nl + p.csize - 1) / p.csize) + kSlice - 1) / kSlice) * kSlice;
+  const int range_beg = min(kbe + nl, c * span);
+  const int range_end = min(kbe + nl, range_beg + span);
 
   const uint16_t* pk_base = p.packed_k + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
   const uint16_t* pv_base = p.packed_v + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
@@ -138,19 +140,19 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const int nslices = (ntok + kSlice - 1) / kSlice;
   // warp w streams slices w, w + kDecWarps, ... of the range, so the CTA walks memory front to back
   const int nmine = nslices > warp ? (nslices - warp + kDecWarps - 1) / kDecWarps : 0;
-  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] - kb;   // indexed by list position
+  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] - kbe;   // indexed by list position
   // Lane r (and r + 16) holds the local index of row r of the warp's j-th slice, read one slice ahead.
   auto fetch_idx = [&](int j) -> int {
     const int li = (warp + j * kDecWarps) * kSlice + (lane & 15);
     const int pos = pos_beg + li;
-    return (j < nmine && li < ntok && pos >= kb) ? __ldg(idx_base + pos) : 0;
+    return (j < nmine && li < ntok && pos >= kbe) ? __ldg(idx_base + pos) : 0;
   };
   auto load_slice = [&](int j, int buf, int idx_reg) {
     const int li0 = (warp + j * kDecWarps) * kSlice;
     {
       const int li = li0 + (lane & 15), pos = pos_beg + li;
       const bool in_list = li < ntok;
-      const bool ok = in_list && (pos < kb || (idx_reg >= 0 && idx_reg < nseq));
+      const bool ok = in_list && (pos < kbe || (idx_reg >= 0 && idx_reg < nseq));
       if (in_list && !ok && lane < 16) raise(p.dev_status, SG_ERR_INDEX);
       const uint32_t mask = __ballot_sync(kFull, ok) & 0xffffu;
       if (lane == 0) s_mask[warp * kBuf + buf] = mask;        // bit r: row r holds a real token
@@ -167,7 +169,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       const uint16_t* srcv = p.packed_v;
       int bytes = 0;
       if (li < ntok) {
-        if (pos < kb) {
+        if (pos < kbe) {
           srck = pk_base + (int64_t)pos * D + col * 8;
           srcv = pv_base + (int64_t)pos * D + col * 8;
           bytes = 16;
@@ -445,12 +447,42 @@ size_t decode_workspace_bytes(const sg_shape*, int32_t, int32_t) { return 0; }  
 
 }  // namespace sg
 
+namespace sg {
+namespace {
+sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v, const int32_t* cu_k,
+                        int32_t total_sel, const int32_t* packed_count, const void* local_k, const void* local_v,
+                        const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
+                        float* lse, void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+}
+}  // namespace sg
+
 extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void* packed_k,
                                            const void* packed_v, const int32_t* cu_k, int32_t total_sel,
                                            const void* local_k, const void* local_v, const int32_t* local_idx,
                                            const int32_t* cu_nloc, int32_t total_loc, float softmax_scale,
                                            void* out, float* lse, void* workspace, size_t workspace_bytes,
                                            int32_t* dev_status, void* stream) {
+  return sg::decode_launch(shape, q, packed_k, packed_v, cu_k, total_sel, nullptr, local_k, local_v, local_idx, cu_nloc,
+                           total_loc, softmax_scale, out, lse, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" sg_status sg_sparse_decode_attn_counted(const sg_shape* shape, const void* q, const void* packed_k,
+                                                   const void* packed_v, const int32_t* cu_cap, int32_t total_cap,
+                                                   const int32_t* packed_count, const void* local_k, const void* local_v,
+                                                   const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc,
+                                                   float softmax_scale, void* out, float* lse, int32_t* dev_status,
+                                                   void* stream) {
+  if (!packed_count || !sg::aligned16(packed_count)) return SG_ERR_INVALID;
+  return sg::decode_launch(shape, q, packed_k, packed_v, cu_cap, total_cap, packed_count, local_k, local_v, local_idx,
+                           cu_nloc, total_loc, softmax_scale, out, lse, nullptr, 0, dev_status, stream);
+}
+
+namespace sg {
+namespace {
+sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v, const int32_t* cu_k,
+                        int32_t total_sel, const int32_t* packed_count, const void* local_k, const void* local_v,
+                        const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
+                        float* lse, void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
   using namespace sg;
   sg_status st = check_shape(shape, false);
   if (st != SG_OK) return st;
@@ -476,6 +508,7 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
   p.cu_k = cu_k;
   p.cu_nloc = cu_nloc;
   p.local_idx = local_idx ? local_idx : cu_nloc;
+  p.packed_count = packed_count;
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.dev_status = dev_status;
@@ -524,3 +557,5 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
 #undef SG_LAUNCH_DECODE
   return SG_OK;
 }
+}  // namespace
+}  // namespace sg

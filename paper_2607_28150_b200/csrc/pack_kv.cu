@@ -18,6 +18,7 @@ struct PackParams {
   const int32_t* sel_idx;
   const int32_t* cu;
   const int32_t* cu_k;
+  const int32_t* sel_count;   // [L][B][Hkv] entries selected per row, or null: every entry of the row
   uint16_t* packed_k;
   uint16_t* packed_v;
   int32_t* dev_status;
@@ -36,11 +37,12 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
   const int64_t row0 = (int64_t)blockIdx.x * (kRowsPerPass * kUnroll) + group;
 
   int4 kv[kUnroll][2];
-  bool ok[kUnroll];
+  bool ok[kUnroll], skip[kUnroll];
 #pragma unroll
   for (int u = 0; u < kUnroll; ++u) {
     const int64_t r = row0 + (int64_t)u * kRowsPerPass;
     ok[u] = false;
+    skip[u] = false;
     kv[u][0] = make_int4(0, 0, 0, 0);
     kv[u][1] = make_int4(0, 0, 0, 0);
     if (r < p.total_rows) {
@@ -54,6 +56,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
       const int j = rem - g * kb;
       const int c0 = p.cu[b];
       const int n = p.cu[b + 1] - c0;
+      if (p.sel_count && j >= p.sel_count[(l * p.B + b) * p.Hkv + g]) { skip[u] = true; continue; }   // not selected: slot left as it is
       const int t = p.sel_idx[(l * p.Hkv + g) * (int64_t)p.K_tot + ck + j];
       if (t >= 0 && t < n) {
         ok[u] = true;
@@ -68,7 +71,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
 #pragma unroll
   for (int u = 0; u < kUnroll; ++u) {
     const int64_t r = row0 + (int64_t)u * kRowsPerPass;
-    if (r < p.total_rows) {
+    if (r < p.total_rows && !skip[u]) {
       const int64_t dst = r * D + lane_in_row * 8;
       __stcs(reinterpret_cast<int4*>(p.packed_k + dst), kv[u][0]);
       __stcs(reinterpret_cast<int4*>(p.packed_v + dst), kv[u][1]);
@@ -80,9 +83,33 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
 }  // namespace
 }  // namespace sg
 
+namespace sg {
+namespace {
+sg_status pack_kv_launch(const sg_shape* shape, const void* k_cache, const void* v_cache, const int32_t* sel_idx,
+                         const int32_t* cu_k, int32_t total_sel, const int32_t* sel_count, void* packed_k, void* packed_v,
+                         int32_t* dev_status, void* stream);
+}
+}  // namespace sg
+
 extern "C" sg_status sg_pack_kv(const sg_shape* shape, const void* k_cache, const void* v_cache,
                                 const int32_t* sel_idx, const int32_t* cu_k, int32_t total_sel,
                                 void* packed_k, void* packed_v, int32_t* dev_status, void* stream) {
+  return sg::pack_kv_launch(shape, k_cache, v_cache, sel_idx, cu_k, total_sel, nullptr, packed_k, packed_v, dev_status, stream);
+}
+
+extern "C" sg_status sg_pack_kv_counted(const sg_shape* shape, const void* k_cache, const void* v_cache,
+                                        const int32_t* sel_idx, const int32_t* cu_cap, int32_t total_cap,
+                                        const int32_t* sel_count, void* packed_k, void* packed_v, int32_t* dev_status,
+                                        void* stream) {
+  if (!sel_count || !sg::aligned16(sel_count)) return SG_ERR_INVALID;
+  return sg::pack_kv_launch(shape, k_cache, v_cache, sel_idx, cu_cap, total_cap, sel_count, packed_k, packed_v, dev_status, stream);
+}
+
+namespace sg {
+namespace {
+sg_status pack_kv_launch(const sg_shape* shape, const void* k_cache, const void* v_cache, const int32_t* sel_idx,
+                         const int32_t* cu_k, int32_t total_sel, const int32_t* sel_count, void* packed_k, void* packed_v,
+                         int32_t* dev_status, void* stream) {
   using namespace sg;
   sg_status st = check_shape(shape, false);
   if (st != SG_OK) return st;
@@ -98,6 +125,7 @@ extern "C" sg_status sg_pack_kv(const sg_shape* shape, const void* k_cache, cons
   p.sel_idx = sel_idx;
   p.cu = shape->cu_seqlens;
   p.cu_k = cu_k;
+  p.sel_count = sel_count;
   p.packed_k = static_cast<uint16_t*>(packed_k);
   p.packed_v = static_cast<uint16_t*>(packed_v);
   p.dev_status = dev_status;
@@ -124,3 +152,5 @@ extern "C" sg_status sg_pack_kv(const sg_shape* shape, const void* k_cache, cons
   SG_CUDA_TRY(cudaGetLastError());
   return SG_OK;
 }
+}  // namespace
+}  // namespace sg
