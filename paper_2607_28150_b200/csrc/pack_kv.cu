@@ -28,7 +28,8 @@ struct PackParams {
   int32_t K_tot, B, Hkv;
 };
 
-template <int D>
+// kCounted: rows beyond a head's count (PackParams::sel_count) are skipped; the plain instantiation carries none of it.
+template <int D, bool kCounted>
 __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams p) {
   constexpr int kTPR = D / 8;                       // threads per row, 16 bytes each
   constexpr int kRowsPerPass = kPackThreads / kTPR;
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
       const int j = rem - g * kb;
       const int c0 = p.cu[b];
       const int n = p.cu[b + 1] - c0;
-      if (p.sel_count && j >= p.sel_count[(l * p.B + b) * p.Hkv + g]) { skip[u] = true; continue; }   // not selected: slot left as it is
+      if (kCounted && j >= p.sel_count[(l * p.B + b) * p.Hkv + g]) { skip[u] = true; continue; }   // not selected: slot left as it is
       const int t = p.sel_idx[(l * p.Hkv + g) * (int64_t)p.K_tot + ck + j];
       if (t >= 0 && t < n) {
         ok[u] = true;
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(kPackThreads) pack_kv_kernel(const PackParams 
 #pragma unroll
   for (int u = 0; u < kUnroll; ++u) {
     const int64_t r = row0 + (int64_t)u * kRowsPerPass;
-    if (r < p.total_rows && !skip[u]) {
+    if (r < p.total_rows && !(kCounted && skip[u])) {
       const int64_t dst = r * D + lane_in_row * 8;
       __stcs(reinterpret_cast<int4*>(p.packed_k + dst), kv[u][0]);
       __stcs(reinterpret_cast<int4*>(p.packed_v + dst), kv[u][1]);
@@ -142,12 +143,14 @@ sg_status pack_kv_launch(const sg_shape* shape, const void* k_cache, const void*
     const int64_t rows_per_cta = (kPackThreads / 16) * kUnroll;
     const int64_t grid = (p.total_rows + rows_per_cta - 1) / rows_per_cta;
     if (grid > 0x7fffffffLL) return SG_ERR_UNSUPPORTED;
-    pack_kv_kernel<128><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
+    if (sel_count) pack_kv_kernel<128, true><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
+    else pack_kv_kernel<128, false><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
   } else {
     const int64_t rows_per_cta = (kPackThreads / 8) * kUnroll;
     const int64_t grid = (p.total_rows + rows_per_cta - 1) / rows_per_cta;
     if (grid > 0x7fffffffLL) return SG_ERR_UNSUPPORTED;
-    pack_kv_kernel<64><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
+    if (sel_count) pack_kv_kernel<64, true><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
+    else pack_kv_kernel<64, false><<<(unsigned)grid, kPackThreads, 0, s>>>(p);
   }
   SG_CUDA_TRY(cudaGetLastError());
   return SG_OK;
