@@ -203,17 +203,19 @@ def proactive_mask(cu_seqlens, num_blocks: int, layer: int, selected) -> np.ndar
     return mask
 
 
-def push_blocks(src_k, src_v, dst_k, dst_v, cu_seqlens, num_blocks: int, layer: int, selected):
+def push_blocks(src_k, src_v, dst_k, dst_v, cu_seqlens, num_blocks: int, layer: int, selected, kv_mask=None):
     """Online proactive transfer of one layer (Section 4.1): returns copies of dst_k, dst_v ([T][Hkv][d] uint16)
-    with the rows of every selected block of `layer` overwritten by the source cache's rows."""
+    with the rows of every selected block of `layer` overwritten by the source cache's rows; with kv_mask (int8 [T])
+    also a copy of it with the pushed tokens set to 1."""
     cu, sel = _c(cu_seqlens, np.int32), _c(selected, np.int32)
     sk, sv = _c(src_k, np.uint16), _c(src_v, np.uint16)
     dk, dv = _c(dst_k, np.uint16).copy(), _c(dst_v, np.uint16).copy()
     T, Hkv, d = sk.shape
     assert int(cu[-1]) == T and sv.shape == sk.shape == dk.shape == dv.shape
+    km = None if kv_mask is None else _c(kv_mask, np.int8).copy()
     _load().sgo_push_blocks(cu.shape[0] - 1, Hkv, d, num_blocks, _p(cu), layer, _p(sel), sel.shape[0],
-                            _p(sk), _p(sv), _p(dk), _p(dv))
-    return dk, dv
+                            _p(sk), _p(sv), _p(dk), _p(dv), None if km is None else _p(km))
+    return (dk, dv) if km is None else (dk, dv, km)
 
 
 def speculative_delivered(num_layers: int, num_blocks: int, k_r: int, ratio: float, iteration: int) -> int:

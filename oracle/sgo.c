@@ -433,9 +433,12 @@ int64_t sgo_speculative_delivered(int L, int M, int64_t K_r, double ratio, int i
 /* Online proactive transfer of one layer (Section 4.1, "Online KV transfer"): the layer's cache is split into
  * M blocks; every block whose position is among the top-K_r (flat id layer*M + m in `selected`) is written,
  * all KV heads, K and V, to the same token positions of the decode-side cache; nothing else is written.
- * Caches of this layer: uint16 [T][Hkv][d] (dense).  selected int32 [K_r], any order. */
+ * Caches of this layer: uint16 [T][Hkv][d] (dense).  selected int32 [K_r], any order.
+ * kv_mask (int8 [T], may be NULL): "each time a KV block is pushed to the decoding node, the prefill node also
+ * updates the corresponding values in the decoding-side KV mask" (Section 4.2): the tokens of a pushed block get
+ * 1 (locally available); other entries keep their value. */
 int sgo_push_blocks(int B, int Hkv, int d, int M, const int32_t *cu, int layer, const int32_t *selected, int K_r,
-                    const uint16_t *src_k, const uint16_t *src_v, uint16_t *dst_k, uint16_t *dst_v) {
+                    const uint16_t *src_k, const uint16_t *src_v, uint16_t *dst_k, uint16_t *dst_v, int8_t *kv_mask) {
     for (int b = 0; b < B; ++b) {
         const int64_t N = cu[b + 1] - cu[b];
         for (int m = 0; m < M; ++m) {
@@ -451,6 +454,7 @@ int sgo_push_blocks(int B, int Hkv, int d, int M, const int32_t *cu, int layer, 
                     dst_k[row + e] = src_k[row + e];
                     dst_v[row + e] = src_v[row + e];
                 }
+                if (kv_mask) kv_mask[cu[b] + t] = 1;
             }
         }
     }

@@ -165,3 +165,26 @@ def test_push_blocks_more_blocks_than_tokens():
     gk, gv = oracle.push_blocks(sk, sv, dk, dv, cu_of((3,)), 8, 0, np.array([2, 3], dtype=np.int32))   # token 1 -> block 2
     assert np.array_equal(gk[1], sk[1]) and np.array_equal(gk[[0, 2]], dk[[0, 2]])
     assert np.array_equal(gv[1], sv[1]) and np.array_equal(gv[[0, 2]], dv[[0, 2]])
+
+
+def test_push_blocks_updates_the_kv_mask_of_the_pushed_tokens_only():
+    """Section 4.2: pushing a block also sets the decode-side KV mask of its tokens to 1; a mask that starts all-remote (2,
+    with 0 for padding) and receives the pushes of the selected blocks ends up as the proactive mask, padding untouched."""
+    lens, M, L = (50, 9), 8, 4
+    cu = cu_of(lens)
+    T = int(cu[-1])
+    sk, sv, dk, dv = _caches(5, lens, 2, 8)
+    selected = np.array(sorted([2 * M + 1, 2 * M + 7, 3 * M + 0, 0, 5]), dtype=np.int32)
+    for layer in range(L):
+        start = np.full(T, 2, dtype=np.int8)
+        start[[3, 55]] = 0                                       # padding entries
+        _, _, km = oracle.push_blocks(sk, sv, dk, dv, cu, M, layer, selected, kv_mask=start)
+        want = oracle.proactive_mask(cu, M, layer, selected)
+        pushed = want == 1
+        assert np.array_equal(km[pushed], np.ones(pushed.sum(), dtype=np.int8))
+        assert np.array_equal(km[~pushed], start[~pushed])
+    # speculative transfer: pushing the remaining blocks later turns the rest local, nothing is ever set back
+    first = oracle.push_blocks(sk, sv, dk, dv, cu, M, 2, selected, kv_mask=np.full(T, 2, dtype=np.int8))[2]
+    rest = np.setdiff1d(np.arange(L * M, dtype=np.int32), selected)
+    second = oracle.push_blocks(sk, sv, dk, dv, cu, M, 2, rest, kv_mask=first)[2]
+    assert np.all(second == 1)
