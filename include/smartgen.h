@@ -214,7 +214,11 @@ sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const i
  *   as for sg_proactive_mask), the rows of all KV heads are copied from src_k/src_v to the same positions of
  *   dst_k/dst_v.  Both caches are bf16, device, addressed with the shape's strides; the call covers the
  *   shape->num_layers consecutive layers layer, layer + 1, ... (the pointers address the first of them; 1 =
- *   the paper's layer-by-layer push as each layer is offloaded); rows of other blocks are not written.  The network hop is out of scope: the
+ *   the paper's layer-by-layer push as each layer is offloaded); rows of other blocks are not written.
+ *   kv_mask (int8 [shape->num_layers][T], device, may be NULL): the decode-side KV mask of those layers; the
+ *   tokens of every pushed block are set to 1 (Section 4.2: every pushed block is followed by an update of the
+ *   decode-side KV mask), all other entries keep their value (2 = remote, 0 = padding).  The same call with the
+ *   blocks of a speculative transfer (Section 4.3) completes the mask over the decoding iterations.  The network hop is out of scope: the
  *   destination is another HBM buffer.  src and dst must not overlap.
  * sg_speculative_delivered -- speculative transfer (Section 4.3; host arithmetic, no GPU): after the prefill
  *   stage pushed the top-K_r blocks, every decoding iteration delivers the next blocks in the order of their
@@ -231,7 +235,7 @@ sg_status sg_proactive_mask(const sg_shape* shape, int32_t num_blocks, int32_t l
                             int32_t num_selected, int8_t* kv_mask, void* stream);
 sg_status sg_push_blocks(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
                          int32_t num_selected, const void* src_k, const void* src_v, void* dst_k, void* dst_v,
-                         void* stream);
+                         int8_t* kv_mask, void* stream);
 int64_t sg_speculative_delivered(int32_t num_layers, int32_t num_blocks, int64_t k_r, double ratio, int32_t iteration);
 
 /*

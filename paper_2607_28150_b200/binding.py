@@ -81,7 +81,7 @@ _lib.sg_sparse_decode_attn_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _v
 _lib.sg_select_threshold.restype = ctypes.c_int
 _lib.sg_select_threshold.argtypes = [_sp, _vp, _f, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.sg_push_blocks.restype = ctypes.c_int
-_lib.sg_push_blocks.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.sg_push_blocks.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_split_index.restype = ctypes.c_int
 _lib.sg_split_index.argtypes = [_sp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn.restype = ctypes.c_int
@@ -326,16 +326,19 @@ def sg_sparse_decode_attn_counted(shape: Shape, q: torch.Tensor, packed_k: Optio
 
 
 def sg_push_blocks(shape: Shape, num_blocks: int, layer: int, selected: Optional[torch.Tensor], src_k: torch.Tensor,
-                   src_v: torch.Tensor, dst_k: torch.Tensor, dst_v: torch.Tensor, stream=None) -> None:
+                   src_v: torch.Tensor, dst_k: torch.Tensor, dst_v: torch.Tensor, kv_mask: Optional[torch.Tensor] = None,
+                   stream=None) -> None:
     """Online proactive transfer: copy the rows (all KV heads, K and V) of every selected block of the layers
     `layer` .. `layer + shape.num_layers - 1` from the source cache to the same positions of the destination
-    cache (the tensors start at `layer`); other rows are untouched."""
+    cache (the tensors start at `layer`); other rows are untouched.  With `kv_mask` (int8 [layers][T]) the pushed
+    tokens are also marked local (1) in the decode-side KV mask."""
     _check(selected, torch.int32, "selected", True)
     for name, t in (("src_k", src_k), ("src_v", src_v), ("dst_k", dst_k), ("dst_v", dst_v)):
         _check(t, _BF16, name)
+    _check(kv_mask, torch.int8, "kv_mask", True)
     n = 0 if selected is None else selected.numel()
     rc = _lib.sg_push_blocks(ctypes.byref(shape), num_blocks, layer, _ptr(selected), n, _ptr(src_k), _ptr(src_v),
-                             _ptr(dst_k), _ptr(dst_v), _stream(stream))
+                             _ptr(dst_k), _ptr(dst_v), _ptr(kv_mask), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_push_blocks")
 

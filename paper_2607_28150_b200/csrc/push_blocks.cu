@@ -7,7 +7,8 @@
 // selected or holds no token of the sequence -- unselected blocks cost no cache traffic.  Otherwise one
 // group of d/8 threads moves one (token, head) row with 16-byte vectors, a warp covers whole 128-byte
 // lines, and each group has kUnroll independent rows (2*kUnroll loads) in flight before the first store.
-// The rows of a block form one contiguous run when the cache is dense.
+// The rows of a block form one contiguous run when the cache is dense.  Optionally the same CTA marks the
+// block's tokens as local (1) in the decode-side KV mask, the update the paper sends behind every pushed block.
 #include "common.cuh"
 
 namespace sg {
@@ -23,6 +24,8 @@ struct PushParams {
   uint16_t* dst_v;
   const int32_t* cu;
   const int32_t* selected;
+  int8_t* kv_mask;         // [layers][T] decode-side KV mask to update (1 = local) for the pushed tokens, or null
+  int64_t T;
   int64_t ls, ts, hs;
   int32_t B, Hkv, M, layer, K_r;
 };
@@ -43,6 +46,8 @@ __global__ void __launch_bounds__(kPushThreads) push_blocks_kernel(const PushPar
   // tokens t with floor(t * M / N) == m
   const int64_t t0 = ((int64_t)m * N + p.M - 1) / p.M, t1 = ((int64_t)(m + 1) * N + p.M - 1) / p.M;
   const int rows = (int)(t1 - t0) * p.Hkv;
+  if (p.kv_mask)                                    // the pushed tokens are locally available from now on
+    for (int t = threadIdx.x; t < (int)(t1 - t0); t += kPushThreads) p.kv_mask[(int64_t)l * p.T + c0 + t0 + t] = 1;
   const int lane_in_row = threadIdx.x % kTPR;
   const int group = threadIdx.x / kTPR;
   const int64_t base = (int64_t)l * p.ls + (c0 + t0) * p.ts + lane_in_row * 8;
@@ -75,7 +80,7 @@ __global__ void __launch_bounds__(kPushThreads) push_blocks_kernel(const PushPar
 
 extern "C" sg_status sg_push_blocks(const sg_shape* shape, int32_t num_blocks, int32_t layer, const int32_t* selected,
                                     int32_t num_selected, const void* src_k, const void* src_v, void* dst_k, void* dst_v,
-                                    void* stream) {
+                                    int8_t* kv_mask, void* stream) {
   using namespace sg;
   sg_status st = check_shape(shape, false);
   if (st != SG_OK) return st;
@@ -92,6 +97,8 @@ extern "C" sg_status sg_push_blocks(const sg_shape* shape, int32_t num_blocks, i
   p.dst_v = static_cast<uint16_t*>(dst_v);
   p.cu = shape->cu_seqlens;
   p.selected = selected;
+  p.kv_mask = kv_mask;
+  p.T = shape->total_tokens;
   p.ls = shape->cache_layer_stride;
   p.ts = shape->cache_token_stride;
   p.hs = shape->cache_head_stride;

@@ -96,3 +96,36 @@ def test_push_blocks_several_layers_in_one_call():
         else:
             want_k, want_v = dk[layer], dv[layer]
         assert np.array_equal(got_k[layer], want_k) and np.array_equal(got_v[layer], want_v)
+
+
+def test_push_blocks_updates_the_kv_mask():
+    """The pushed tokens become local (1) in the decode-side KV mask, every other entry (remote 2, padding 0) keeps its
+    value; several layers in one call; pushing the remaining blocks afterwards completes the mask."""
+    import torch
+    import gpu_ops
+    import paper_2607_28150_b200.binding as sg
+    rng = np.random.default_rng(11)
+    lens, Hkv, d, M, L = (900, 333, 5), 2, 64, 24, 4
+    cu = cu_of(lens); T = int(cu[-1])
+    selected = np.sort(rng.choice(L * M, size=40, replace=False)).astype(np.int32)
+    mk = lambda: rng.integers(0, 1 << 16, size=(L, T, Hkv, d), dtype=np.uint16)
+    sk, sv, dk, dv = mk(), mk(), mk(), mk()
+    start = np.full((L, T), 2, dtype=np.int8)
+    start[:, [7, 901, T - 1]] = 0
+    shpL = gpu_ops.shape_of(L, Hkv, Hkv, d, 1, cu)
+    gk, gv = gpu_ops.dev(dk), gpu_ops.dev(dv)
+    mask = gpu_ops.Guarded((L, T), torch.int8, 9)
+    mask.view.copy_(torch.from_numpy(start).cuda())
+    sg.sg_push_blocks(shpL, M, 0, gpu_ops.dev(selected), gpu_ops.dev(sk), gpu_ops.dev(sv), gk, gv, kv_mask=mask.view)
+    got_mask = mask.numpy()
+    for layer in range(L):
+        want_k, want_v, want_m = oracle.push_blocks(sk[layer], sv[layer], dk[layer], dv[layer], cu, M, layer, selected, kv_mask=start[layer])
+        assert np.array_equal(got_mask[layer], want_m)
+        assert np.array_equal(gk[layer].cpu().numpy().view(np.uint16), want_k)
+        assert np.array_equal(gv[layer].cpu().numpy().view(np.uint16), want_v)
+    # the speculative transfer delivers the rest: afterwards every token (a pushed padding entry included) is local
+    rest = np.setdiff1d(np.arange(L * M, dtype=np.int32), selected).astype(np.int32)
+    sg.sg_push_blocks(shpL, M, 0, gpu_ops.dev(rest), gpu_ops.dev(sk), gpu_ops.dev(sv), gk, gv, kv_mask=mask.view)
+    final = mask.numpy()
+    assert np.array_equal(final, np.ones_like(start))
+    assert np.array_equal(gk.cpu().numpy().view(np.uint16), sk)
