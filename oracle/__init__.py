@@ -126,12 +126,14 @@ def pack_kv(k_cache: np.ndarray, v_cache: np.ndarray, cu_seqlens: np.ndarray, se
 
 
 def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu_seqlens, local_idx, cu_nloc,
-                       softmax_scale: float = 0.0, packed_count: Optional[np.ndarray] = None):
+                       softmax_scale: float = 0.0, packed_count: Optional[np.ndarray] = None,
+                       local_skip: Optional[np.ndarray] = None):
     """(out float32 [B][H_q][d], lse float32 [B][H_q]) of attention over packed rows ++ indexed local rows.
 
     q uint16 [B][H_q][d]; packed_k/v uint16 [K_tot*H_kv][d]; local_k/v uint16 [T][H_kv][d];
     local_idx int32 [H_kv][NL_tot].  With packed_count (int32 [B][H_kv]) only the first packed_count[b][g] packed rows
-    of each (sequence, KV head) are attended.
+    of each (sequence, KV head) are attended; with local_skip (int32 [B][H_kv]) the first local_skip[b][g] entries of
+    each local-index row are left out.
     """
     q, pk, pv = _c(q, np.uint16), _c(packed_k, np.uint16), _c(packed_v, np.uint16)
     lk, lv = _c(local_k, np.uint16), _c(local_v, np.uint16)
@@ -143,7 +145,8 @@ def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu_seqlens
     lse = np.zeros((B, Hq), dtype=np.float32)
     rc = _load().sgo_sparse_decode_attn(B, Hq, Hkv, d, _p(cu), _p(q), _p(pk), _p(pv), _p(ck), _p(lk), _p(lv),
                                         _i64(Hkv * d), _i64(d), _p(li), _p(cl), ctypes.c_double(softmax_scale),
-                                        _p(out), _p(lse), None if packed_count is None else _p(_c(packed_count, np.int32)))
+                                        _p(out), _p(lse), None if packed_count is None else _p(_c(packed_count, np.int32)),
+                                        None if local_skip is None else _p(_c(local_skip, np.int32)))
     if rc:
         raise RuntimeError("sgo_sparse_decode_attn failed: %d" % rc)
     return out, lse

@@ -217,12 +217,15 @@ int sgo_pack_kv(int L, int B, int Hkv, int d, const int32_t *cu, const uint16_t 
  * An empty list gives out = 0 and lse = -inf.  Returns 3 on an out-of-range local index.
  * packed_count (int32 [B][Hkv], may be NULL): when the selection kept a different number of entries per KV head
  * (threshold selection), only the first packed_count[b][g] of the k_b packed rows of (b, g) are in the list.
+ * local_skip (int32 [B][Hkv], may be NULL): the first local_skip[b][g] entries of the local-index row of (b, g) are
+ * not in the list.  With Algorithm 1's reordered KV index as local_idx (remote entries first) and both arrays set
+ * to the remote counts, the list is [remote rows, fetched and packed] ++ [local rows, by index]: two-lane fetching.
  */
 int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, const uint16_t *q,
                            const uint16_t *packed_k, const uint16_t *packed_v, const int32_t *cu_k,
                            const uint16_t *local_k, const uint16_t *local_v, int64_t ts, int64_t hs,
                            const int32_t *local_idx, const int32_t *cu_nloc, double softmax_scale,
-                           float *out, float *lse, const int32_t *packed_count) {
+                           float *out, float *lse, const int32_t *packed_count, const int32_t *local_skip) {
     if (Hkv <= 0 || Hq % Hkv != 0) return 1;
     const int G = Hq / Hkv;
     const int64_t NL_tot = cu_nloc[B];
@@ -241,7 +244,13 @@ int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, con
                 if (kbe > kb) kbe = kb;
             }
             const int nl = cu_nloc[b + 1] - cu_nloc[b];
-            const int n = kbe + nl;
+            int skip = 0;
+            if (local_skip) {
+                skip = local_skip[(int64_t)b * Hkv + g];
+                if (skip < 0) skip = 0;
+                if (skip > nl) skip = nl;
+            }
+            const int n = kbe + nl - skip;
             float *o = out + ((int64_t)b * Hq + h) * d;
             for (int c = 0; c < d; ++c) o[c] = 0.0f;
             if (lse) lse[(int64_t)b * Hq + h] = -INFINITY;
@@ -256,7 +265,7 @@ int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, con
                 kr[m] = packed_k + row;
                 vr[m] = packed_v + row;
             }
-            for (int j = 0; j < nl; ++j) {
+            for (int j = skip; j < nl; ++j) {
                 const int32_t t = local_idx[(int64_t)g * NL_tot + cu_nloc[b] + j];
                 if (t < 0 || t >= N) { bad = 3; continue; }
                 const int64_t off = ((int64_t)cu[b] + t) * ts + g * hs;

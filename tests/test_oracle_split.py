@@ -69,3 +69,32 @@ def test_mask_footprint_matches_printed_example():
     mask = np.zeros(tokens, dtype=np.int8)            # the mask the oracle indexes: one int8 per token
     assert mask.nbytes == per_layer == 64 * 1024
     assert layers * mask.nbytes / 2**20 == total_mb
+
+
+def test_two_lane_fetching_equals_attention_over_the_kv_index():
+    """Section 4.2 end to end on the oracle: split and reorder the KV index by the KV mask (Algorithm 1), fetch the remote
+    entries into a packed buffer, attend [packed remote rows] ++ [local rows by index]; the result is attention over the
+    KV index set itself (order along the sequence axis does not matter)."""
+    import oracle
+    from helpers import cu_of, rand_bf16
+    rng = np.random.default_rng(8)
+    lens, ks, Hq, Hkv, d = (70, 41), (20, 9), 4, 2, 16
+    cu, ck = cu_of(lens), cu_of(ks)
+    T, Kt = int(cu[-1]), int(ck[-1])
+    k, v = rand_bf16(rng, (1, T, Hkv, d)), rand_bf16(rng, (1, T, Hkv, d))
+    q = rand_bf16(rng, (len(lens), Hq, d))
+    kv_index = np.zeros((Hkv, Kt), dtype=np.int32)
+    for g in range(Hkv):
+        for b, n in enumerate(lens):
+            kv_index[g, ck[b]:ck[b + 1]] = np.sort(rng.choice(n, ks[b], replace=False))
+    kv_mask = rng.choice(np.array([1, 2], dtype=np.int8), size=T)
+    reordered, loc, rem, nl, nr = oracle.split_index(kv_index, kv_mask, cu, ck, reorder=True)
+    assert len(set(nr.ravel().tolist())) > 1
+    # remote lane: the first nr[b][g] entries of every reordered row are fetched and packed (counts per head)
+    pk, pv = oracle.pack_kv(k, v, cu, reordered[None], ck, sel_count=nr[None])
+    # two-lane attention: packed remote rows, then the local rest of the reordered row read by index from the cache
+    out, lse = oracle.sparse_decode_attn(q, pk[0], pv[0], ck, k[0], v[0], cu, reordered, ck, packed_count=nr, local_skip=nr)
+    # reference: everything read by index (one lane)
+    empty = np.zeros((0, d), dtype=np.uint16)
+    want, want_lse = oracle.sparse_decode_attn(q, empty, empty, cu_of((0, 0)), k[0], v[0], cu, kv_index, ck)
+    assert np.allclose(out, want, atol=1e-6) and np.allclose(lse, want_lse, atol=1e-6)
