@@ -269,8 +269,15 @@ sg_status sg_select_threshold(const sg_shape* shape, const float* scores, float 
  *                                 everything else as sg_pack_kv with cu_cap / total_cap in place of cu_k / total_sel.
  *   sg_sparse_decode_attn_counted packed_count int32 [B][H_kv], device (one layer's slice of sel_count): the list of
  *                                 (b, g) is its first packed_count[b][g] packed rows, then its local rows; values
- *                                 are clamped to [0, cap_b].  No workspace.  Everything else as sg_sparse_decode_attn.
- * With every count equal to its cap the two calls are sg_pack_kv and sg_sparse_decode_attn.
+ *                                 are clamped to [0, cap_b].  local_skip int32 [B][H_kv], device: the first
+ *                                 local_skip[b][g] entries of the local-index row of (b, g) are not in the list
+ *                                 (clamped to the row).  Either array may be NULL (not both).  No workspace.
+ *                                 Everything else as sg_sparse_decode_attn.
+ * With every count equal to its cap (and no skip) the two calls are sg_pack_kv and sg_sparse_decode_attn.
+ * Two-lane fetching (Section 4.2) with these calls: sg_split_index with reorder gives, per head, the KV index with
+ * its n_remote[b][g] remote entries first; sg_pack_kv_counted(sel_idx = reordered, sel_count = n_remote) fetches the
+ * remote lane from the prefill-side cache; sg_sparse_decode_attn_counted(packed_count = n_remote, local_idx =
+ * reordered, cu_nloc = cu_k, local_skip = n_remote) attends the fetched rows and the local rest of every row.
  */
 sg_status sg_pack_kv_counted(const sg_shape* shape, const void* k_cache, const void* v_cache, const int32_t* sel_idx,
                              const int32_t* cu_cap, int32_t total_cap, const int32_t* sel_count, void* packed_k,
@@ -278,8 +285,8 @@ sg_status sg_pack_kv_counted(const sg_shape* shape, const void* k_cache, const v
 sg_status sg_sparse_decode_attn_counted(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v,
                                         const int32_t* cu_cap, int32_t total_cap, const int32_t* packed_count,
                                         const void* local_k, const void* local_v, const int32_t* local_idx,
-                                        const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
-                                        float* lse, int32_t* dev_status, void* stream);
+                                        const int32_t* cu_nloc, int32_t total_loc, const int32_t* local_skip,
+                                        float softmax_scale, void* out, float* lse, int32_t* dev_status, void* stream);
 
 /*
  * sg_score_static -- sg_score without a workspace argument, for callers that cannot allocate.

@@ -77,7 +77,7 @@ _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
 _lib.sg_pack_kv_counted.restype = ctypes.c_int
 _lib.sg_pack_kv_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn_counted.restype = ctypes.c_int
-_lib.sg_sparse_decode_attn_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp, _vp]
+_lib.sg_sparse_decode_attn_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _f, _vp, _vp, _vp, _vp]
 _lib.sg_select_threshold.restype = ctypes.c_int
 _lib.sg_select_threshold.argtypes = [_sp, _vp, _f, _vp, _i32, _vp, _vp, _vp, _vp]
 _lib.sg_push_blocks.restype = ctypes.c_int
@@ -305,22 +305,24 @@ def sg_pack_kv_counted(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tenso
 
 
 def sg_sparse_decode_attn_counted(shape: Shape, q: torch.Tensor, packed_k: Optional[torch.Tensor], packed_v: Optional[torch.Tensor],
-                                  cu_cap: torch.Tensor, total_cap: int, packed_count: torch.Tensor,
+                                  cu_cap: torch.Tensor, total_cap: int, packed_count: Optional[torch.Tensor],
                                   local_k: Optional[torch.Tensor], local_v: Optional[torch.Tensor],
                                   local_idx: Optional[torch.Tensor], cu_nloc: torch.Tensor, total_loc: int, out: torch.Tensor,
                                   lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
-                                  dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+                                  dev_status: Optional[torch.Tensor] = None, stream=None,
+                                  local_skip: Optional[torch.Tensor] = None) -> None:
     """sg_sparse_decode_attn for per-head counts: of the cap_b packed rows of (b, g) only the first packed_count[b][g]
-    are attended."""
+    are attended, and the first local_skip[b][g] entries of its local-index row are left out."""
     _check(q, _BF16, "q"); _check(out, _BF16, "out"); _check(cu_cap, torch.int32, "cu_cap"); _check(cu_nloc, torch.int32, "cu_nloc")
-    _check(packed_count, torch.int32, "packed_count")
+    _check(packed_count, torch.int32, "packed_count", True); _check(local_skip, torch.int32, "local_skip", True)
     _check(packed_k, _BF16, "packed_k", True); _check(packed_v, _BF16, "packed_v", True)
     _check(local_k, _BF16, "local_k", True); _check(local_v, _BF16, "local_v", True)
     _check(local_idx, torch.int32, "local_idx", True); _check(lse, torch.float32, "lse", True)
     _check(dev_status, torch.int32, "dev_status", True)
     rc = _lib.sg_sparse_decode_attn_counted(ctypes.byref(shape), _ptr(q), _ptr(packed_k), _ptr(packed_v), _ptr(cu_cap), total_cap,
                                             _ptr(packed_count), _ptr(local_k), _ptr(local_v), _ptr(local_idx), _ptr(cu_nloc),
-                                            total_loc, softmax_scale, _ptr(out), _ptr(lse), _ptr(dev_status), _stream(stream))
+                                            total_loc, _ptr(local_skip), softmax_scale, _ptr(out), _ptr(lse), _ptr(dev_status),
+                                            _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_sparse_decode_attn_counted")
 

@@ -41,6 +41,7 @@ struct DecParams {
   const int32_t* cu_nloc;
   const int32_t* local_idx;
   const int32_t* packed_count;   // [B][Hkv] packed rows of a (sequence, KV head) that are in the list, or null: all k_b
+  const int32_t* local_skip;     // [B][Hkv] leading entries of the head's local-index row that are not in the list, or null
   uint16_t* out;
   float* lse;
   int32_t* dev_status;
@@ -121,7 +122,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
   const int kb = p.cu_k[b + 1] - p.cu_k[b];                    // packed rows per KV head (the slot size in the buffer)
   const int kbe = p.packed_count ? min(kb, max(0, __ldg(p.packed_count + (int64_t)b * p.Hkv + g))) : kb;   // ... of which in the list
-  const int nl = p.cu_nloc[b + 1] - p.cu_nloc[b];
+  const int nl_row = p.cu_nloc[b + 1] - p.cu_nloc[b];
+  const int lskip = p.local_skip ? min(nl_row, max(0, __ldg(p.local_skip + (int64_t)b * p.Hkv + g))) : 0;
+  const int nl = nl_row - lskip;
   const int c0 = p.cu[b];
   const int nseq = p.cu[b + 1] - c0;
   // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
@@ -140,7 +143,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const int nslices = (ntok + kSlice - 1) / kSlice;
   // warp w streams slices w, w + kDecWarps, ... of the range, so the CTA walks memory front to back
   const int nmine = nslices > warp ? (nslices - warp + kDecWarps - 1) / kDecWarps : 0;
-  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] - kbe;   // indexed by list position
+  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + lskip - kbe;   // indexed by list position
   // Lane r (and r + 16) holds the local index of row r of the warp's j-th slice, read one slice ahead.
   auto fetch_idx = [&](int j) -> int {
     const int li = (warp + j * kDecWarps) * kSlice + (lane & 15);
@@ -450,9 +453,10 @@ size_t decode_workspace_bytes(const sg_shape*, int32_t, int32_t) { return 0; }  
 namespace sg {
 namespace {
 sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v, const int32_t* cu_k,
-                        int32_t total_sel, const int32_t* packed_count, const void* local_k, const void* local_v,
-                        const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
-                        float* lse, void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream);
+                        int32_t total_sel, const int32_t* packed_count, const int32_t* local_skip, const void* local_k,
+                        const void* local_v, const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc,
+                        float softmax_scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                        int32_t* dev_status, void* stream);
 }
 }  // namespace sg
 
@@ -462,27 +466,28 @@ extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q,
                                            const int32_t* cu_nloc, int32_t total_loc, float softmax_scale,
                                            void* out, float* lse, void* workspace, size_t workspace_bytes,
                                            int32_t* dev_status, void* stream) {
-  return sg::decode_launch(shape, q, packed_k, packed_v, cu_k, total_sel, nullptr, local_k, local_v, local_idx, cu_nloc,
-                           total_loc, softmax_scale, out, lse, workspace, workspace_bytes, dev_status, stream);
+  return sg::decode_launch(shape, q, packed_k, packed_v, cu_k, total_sel, nullptr, nullptr, local_k, local_v, local_idx,
+                           cu_nloc, total_loc, softmax_scale, out, lse, workspace, workspace_bytes, dev_status, stream);
 }
 
 extern "C" sg_status sg_sparse_decode_attn_counted(const sg_shape* shape, const void* q, const void* packed_k,
                                                    const void* packed_v, const int32_t* cu_cap, int32_t total_cap,
                                                    const int32_t* packed_count, const void* local_k, const void* local_v,
                                                    const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc,
-                                                   float softmax_scale, void* out, float* lse, int32_t* dev_status,
-                                                   void* stream) {
-  if (!packed_count || !sg::aligned16(packed_count)) return SG_ERR_INVALID;
-  return sg::decode_launch(shape, q, packed_k, packed_v, cu_cap, total_cap, packed_count, local_k, local_v, local_idx,
-                           cu_nloc, total_loc, softmax_scale, out, lse, nullptr, 0, dev_status, stream);
+                                                   const int32_t* local_skip, float softmax_scale, void* out, float* lse,
+                                                   int32_t* dev_status, void* stream) {
+  if ((!packed_count && !local_skip) || !sg::aligned16(packed_count) || !sg::aligned16(local_skip)) return SG_ERR_INVALID;
+  return sg::decode_launch(shape, q, packed_k, packed_v, cu_cap, total_cap, packed_count, local_skip, local_k, local_v,
+                           local_idx, cu_nloc, total_loc, softmax_scale, out, lse, nullptr, 0, dev_status, stream);
 }
 
 namespace sg {
 namespace {
 sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v, const int32_t* cu_k,
-                        int32_t total_sel, const int32_t* packed_count, const void* local_k, const void* local_v,
-                        const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc, float softmax_scale, void* out,
-                        float* lse, void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
+                        int32_t total_sel, const int32_t* packed_count, const int32_t* local_skip, const void* local_k,
+                        const void* local_v, const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc,
+                        float softmax_scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                        int32_t* dev_status, void* stream) {
   using namespace sg;
   sg_status st = check_shape(shape, false);
   if (st != SG_OK) return st;
@@ -509,6 +514,7 @@ sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed
   p.cu_nloc = cu_nloc;
   p.local_idx = local_idx ? local_idx : cu_nloc;
   p.packed_count = packed_count;
+  p.local_skip = local_skip;
   p.out = static_cast<uint16_t*>(out);
   p.lse = lse;
   p.dev_status = dev_status;

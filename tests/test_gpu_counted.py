@@ -97,3 +97,52 @@ def test_counts_equal_to_the_caps_reproduce_the_plain_calls():
                                      gpu_ops.dev(k[0]), gpu_ops.dev(v[0]), None, gpu_ops.dev(cl), 0, out_b, lse_b)
     assert np.array_equal(bf16_bits_to_f32(out_b.cpu().numpy().view(np.uint16)), out_a)
     assert np.array_equal(lse_b.cpu().numpy(), lse_a)
+
+
+@pytest.mark.parametrize("lens,ks,Hq,Hkv,d,remote_share", [
+    ((8192,), (820,), 32, 8, 128, 0.34),                      # 8B-shaped layer, the paper's on-demand ratio
+    ((300, 64, 5000, 77), (37, 64, 1000, 5), 32, 8, 128, 0.5),
+    (tuple(120 + 11 * i for i in range(40)), tuple(10 + i for i in range(40)), 16, 8, 64, 0.2),
+    ((2000,), (333,), 32, 2, 128, 1.0),                       # everything remote
+    ((2000,), (333,), 32, 2, 128, 0.0),                       # everything local
+])
+def test_two_lane_fetching_on_the_gpu(lens, ks, Hq, Hkv, d, remote_share):
+    """Section 4.2 end to end through the C ABI: Algorithm 1 (split + reorder) -> fetch the remote lane into a packed
+    buffer with per-head counts -> attend [packed remote rows] ++ [local rest of the row, by index].  Equals the oracle's
+    attention over the KV index set read in one lane."""
+    import torch
+    import gpu_ops
+    import paper_2607_28150_b200.binding as sg
+    rng = np.random.default_rng(4)
+    B = len(lens)
+    cu, ck = cu_of(lens), cu_of(ks)
+    T, Kt = int(cu[-1]), int(ck[-1])
+    k, v = rand_bf16(rng, (1, T, Hkv, d)), rand_bf16(rng, (1, T, Hkv, d))
+    q = rand_bf16(rng, (B, Hq, d))
+    kv_index = np.zeros((Hkv, Kt), dtype=np.int32)
+    for g in range(Hkv):
+        for b, n in enumerate(lens):
+            kv_index[g, ck[b]:ck[b + 1]] = np.sort(rng.choice(n, ks[b], replace=False))
+    kv_mask = np.where(rng.random(T) < remote_share, 2, 1).astype(np.int8)
+    shp = gpu_ops.shape_of(1, Hq, Hkv, d, 1, cu)
+    st = gpu_ops.status_word()
+    d_idx, d_ck = gpu_ops.dev(kv_index), gpu_ops.dev(ck)
+    reo = torch.empty_like(d_idx); loc = torch.empty_like(d_idx); rem = torch.empty_like(d_idx)
+    nl = torch.empty((B, Hkv), dtype=torch.int32, device="cuda"); nr = torch.empty_like(nl)
+    sg.sg_split_index(shp, d_idx, d_ck, Kt, gpu_ops.dev(kv_mask), True, reo, loc, rem, nl, nr, st)
+    # remote lane: fetch the first n_remote entries of every reordered row from the prefill-side cache
+    pk = torch.zeros((1, Kt * Hkv, d), dtype=torch.int16, device="cuda"); pv = torch.zeros_like(pk)
+    d_k, d_v = gpu_ops.dev(k), gpu_ops.dev(v)
+    sg.sg_pack_kv_counted(shp, d_k, d_v, reo.unsqueeze(0).contiguous(), d_ck, Kt, nr.unsqueeze(0).contiguous(), pk, pv, st)
+    # both lanes
+    out = gpu_ops.Guarded((B, Hq, d), torch.int16, 0x5555)
+    lse = gpu_ops.Guarded((B, Hq), torch.float32, -7.0)
+    sg.sg_sparse_decode_attn_counted(shp, gpu_ops.dev(q), pk[0], pv[0], d_ck, Kt, nr, d_k[0], d_v[0], reo, d_ck, Kt,
+                                     out.view, lse.view, 0.0, st, local_skip=nr)
+    got_o, got_l = bf16_bits_to_f32(out.numpy()), lse.numpy()
+    assert gpu_ops.read_status(st) == 0
+    empty = np.zeros((0, d), dtype=np.uint16)
+    want_o, want_l = oracle.sparse_decode_attn(q, empty, empty, cu_of((0,) * B), k[0], v[0], cu, kv_index, ck)
+    assert np.abs(got_o - want_o).max() <= 2e-2 and np.abs(got_l - want_l).max() <= 1e-3
+    n_remote = nr.cpu().numpy()
+    assert n_remote.sum() == int((kv_mask[np.concatenate([cu[b] + kv_index[:, ck[b]:ck[b + 1]].ravel() for b in range(B)])] == 2).sum())
