@@ -542,6 +542,11 @@ def run_ours(args):
     }
     roofs["score"]["tensor_tflops"] = work["score"]["flops"] / (st["score"] * 1e-3) / 1e12
     roofs["score"]["tensor_frac_of_sustained"] = roofs["score"]["tensor_tflops"] / tc_peak
+    # third ceiling of the scoring kernel: one exp2 per score element and pass on the SFU (16 per clock and SM)
+    exps = 2.0 * work["score"]["flops"] / (2.0 * cfg.head_dim)
+    sfu_peak = 16.0 * 148 * 1.965e9
+    roofs["score"]["sfu_exp_per_s"] = exps / (st["score"] * 1e-3)
+    roofs["score"]["sfu_frac_at_max_clock"] = roofs["score"]["sfu_exp_per_s"] / sfu_peak
     R = cfg.group * W
     if R > peaks["bf16_tflops_sustained"] * 1e3 / peaks["hbm_gbs"]:       # above the ridge: tensor cores bind
         roofs["score"].update(bound="tensor", achieved=roofs["score"]["tensor_tflops"], peak=tc_peak, unit="TFLOP/s",
