@@ -41,6 +41,7 @@ constexpr int kScoreThreads = 64 + kEpiThreads;   // warp 0: TMA, warp 1: MMA + 
 constexpr int kTileKeys = 128;
 constexpr int kRing = 4 / kEpiGroups;        // accumulator stages per epilogue warpgroup
 constexpr int kAccStages = 4;             // 4 x 128 fp32 columns = the whole 512-column TMEM
+constexpr int kPartSlots = 8;             // pass 2, several row blocks per key tile: partial column sums of up to 8 tiles in flight
 constexpr uint32_t kTmemCols = 512;
 constexpr int kMaxKStages = 4;
 constexpr int kSmemLimit = 232448;        // 227 KB opt-in dynamic shared memory per CTA
@@ -271,8 +272,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 28 * 8 + 4);
   float* lse_buf = reinterpret_cast<float*>(tail + 240);              // [Ralloc] row log-sum-exps of the current pass-2 item
   float* sm_stat = lse_buf + p.Ralloc;                            // pass 1: m[groups][Ralloc], l[groups][Ralloc]
-  float* sm_part = sm_stat + 2 * kEpiGroups * p.Ralloc;               // pass 2, several blocks per tile: [2][groups][128] partial column sums
-  int* s_cu = reinterpret_cast<int*>(sm_part + 2 * kEpiGroups * 128);         // [B+1]
+  float* sm_part = sm_stat + 2 * kEpiGroups * p.Ralloc;               // pass 2, several blocks per tile: [kPartSlots][groups][128] partial column sums
+  const int part_slots = p.Rpad > 384 ? 4 : (p.Rpad > 128 ? 8 : 0);   // tiles in flight (see the pass-2 combine)
+  int* sm_cnt = reinterpret_cast<int*>(sm_part + part_slots * kEpiGroups * 128);   // [kPartSlots][4 lane quarters] partials written
+  int* s_cu = sm_cnt + kPartSlots * 4;                                // [B+1]
   int* s_prefix = s_cu + p.B + 1;                                     // [B+1]
 
   auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
@@ -291,6 +294,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     for (int s = 0; s < kMaxKStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
     for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), 4); }
     *abort_flag = 0;
+    for (int i = 0; i < kPartSlots * 4; ++i) sm_cnt[i] = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
@@ -590,8 +594,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
           const int rmin = (t - first_win) * p.G;        // rows below rmin cannot see key t
           float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          const uint32_t n0 = tile_count;                // running block count at the start of this tile
+          bool mine = false;                             // this warpgroup drains at least one block of the tile
           for (int blk = 0; blk < nblk; ++blk) {
             if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+            mine = true;
             const int as = wg * kRing + ring;
             if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
             if (!ok) continue;
@@ -630,14 +637,28 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           }
           float total = (a0 + a1) + (a2 + a3);
           if (blockwise) {
-            // the tile's column blocks were dealt to different warpgroups: add their partial column sums
-            float* part = sm_part + (tile & 1) * (kEpiGroups * 128);
+            // The tile's row blocks were dealt to different warpgroups.  Each warpgroup that had one leaves its partial
+            // column sums in shared memory; per lane quarter, the warp that writes the last partial adds them up in a
+            // fixed order (bitwise reproducible) and stores the importance -- no block-wide barrier per tile.  A slot
+            // is reused S tiles later: block m is issued only after blocks m-4 .. m-7 were released, and the
+            // warpgroups that released them had finished everything up to block m-8; with (S-1)*nblk >= 7 all
+            // partials of the slot's previous tile are summed before the slot is written again.
+            if (!mine) continue;
+            const int nwg = nblk < kEpiGroups ? nblk : kEpiGroups;      // warpgroups that drain blocks of this tile
+            const int slot = tile & (nblk >= 4 ? 3 : 7);
+            float* part = sm_part + slot * (kEpiGroups * 128);
             part[wg * 128 + row_in_tile] = total;
-            epi_bar_sync();
-            if (wg != 0) continue;
+            __threadfence_block();
+            __syncwarp();
+            int old = 0;
+            if (lane == 0) old = atomicAdd(&sm_cnt[slot * 4 + lane_grp], 1);
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if (old != nwg - 1) continue;
+            __threadfence_block();
             total = 0.f;
-#pragma unroll
-            for (int w = 0; w < kEpiGroups; ++w) total += part[w * 128 + row_in_tile];
+            for (int i = 0; i < nwg; ++i) total += part[((n0 + i) % kEpiGroups) * 128 + row_in_tile];
+            __syncwarp();
+            if (lane == 0) sm_cnt[slot * 4 + lane_grp] = 0;
           }
           if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
         }
@@ -687,7 +708,8 @@ ScorePlan plan_score(const sg_shape* s) {
   pl.Ralloc = (pl.R + 127) & ~127;
   const int q_bytes = pl.Ralloc * D * 2;
   const int k_stage = kTileKeys * D * 2;
-  const int tail = (240 + (1 + 2 * kEpiGroups) * pl.Ralloc * 4 + 2 * kEpiGroups * 128 * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
+  const int part_slots = pl.Rpad > 384 ? 4 : (pl.Rpad > 128 ? 8 : 0);
+  const int tail = (240 + (1 + 2 * kEpiGroups) * pl.Ralloc * 4 + part_slots * kEpiGroups * 128 * 4 + kPartSlots * 4 * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
   const int avail = kSmemLimit - 1024 - tail;
   // Two Q buffers let the next item's queries load while the current item computes; fall back to one
   // when that would leave fewer than three K stages.
