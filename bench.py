@@ -539,7 +539,7 @@ def run_ours(args):
     ms_step, st = timed(False, args.steps, max(3, args.warmup))
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     ms_e2e, st_e = timed(True, e2e_steps, 1)
-    ms_pipe = e2e_pipelined_ms() if world == 1 else None
+    ms_pipe = e2e_pipelined_ms() if world == 1 and not args.no_extras else None
     clocks = sampler.stop() if rank == 0 else {}       # sampled over both timed regions
     status = hp.read_status()
 
@@ -603,10 +603,10 @@ def run_ours(args):
                "score_tflops": work["score"]["flops"] * fr / t["score"] / 1e12}
 
     kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
-    next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 else None
-    layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 else None
+    next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 and not args.no_extras else None
+    layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
     sweep = None
-    if args.workload == "c2" and not args.no_decode_sweep and world == 1:
+    if args.workload == "c2" and not args.no_decode_sweep and not args.no_extras and world == 1:
         del d_k, d_v, h_k, h_v
         torch.cuda.empty_cache()
         sweep = decode_sweep_points(dev, peaks)
@@ -653,6 +653,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-sweep", action="store_true", help="skip the extra decode-only points (c2 only)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="only the timed step: skip the decode sweep, the timings of the other entry points, the "
+                         "layer-by-layer prefill and the pipelined e2e (for profiling the step itself)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
