@@ -574,6 +574,8 @@ def run_ours(args):
     }
     roofs["score"]["tensor_tflops"] = work["score"]["flops"] / (st["score"] * 1e-3) / 1e12
     roofs["score"]["tensor_frac_of_sustained"] = roofs["score"]["tensor_tflops"] / tc_peak
+    roofs["select"]["rows"] = L * B * Hkv
+    roofs["select"]["us_per_row_amortised"] = 1e3 * st["select"] / max(1, L * B * Hkv)
     # third ceiling of the scoring kernel: one exp2 per score element and pass on the SFU (16 per clock and SM)
     exps = 2.0 * work["score"]["flops"] / (2.0 * cfg.head_dim)
     sfu_peak = 16.0 * 148 * 1.965e9
