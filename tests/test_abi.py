@@ -61,3 +61,42 @@ def test_host_side_argument_checks_need_no_gpu():
     # score: more rows per KV head than the shared-memory Q buffer holds is refused, not truncated
     big = sg.Shape(1, 1, 64, 2, 128, 64, 16384, 16384, 0x1000, 16384 * 256, 256, 128)      # G*W = 2048
     assert lib.sg_score(ctypes.byref(big), fake, fake, fake, fake, 1 << 30, None, None) == sg.SG_ERR_UNSUPPORTED
+
+
+def test_header_is_plain_c_and_a_c_program_links_against_the_library(tmp_path):
+    """The boundary is usable from C: the header compiles as C99 (and C++11) with warnings on, and a C program that
+    only uses host-side calls links against the shared library and runs without a GPU."""
+    import shutil
+    import subprocess
+    hdr = os.path.join(ROOT, "include", "smartgen.h")
+    if shutil.which("gcc") is None:
+        return
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr], check=True)
+    if shutil.which("g++"):
+        subprocess.run(["g++", "-std=c++11", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr], check=True)
+    src = tmp_path / "caller.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "smartgen.h"
+int main(void) {
+  sg_shape s;
+  memset(&s, 0, sizeof s);
+  /* a null cu_seqlens is rejected on the host, before anything touches a device */
+  s.num_layers = 1; s.batch = 1; s.num_q_heads = 8; s.num_kv_heads = 2; s.head_dim = 128; s.window = 4;
+  s.total_tokens = 16; s.max_seqlen = 16; s.cache_layer_stride = 16 * 256; s.cache_token_stride = 256; s.cache_head_stride = 128;
+  if (sg_pack_kv(&s, 0, 0, 0, 0, 4, 0, 0, 0, 0) != SG_ERR_INVALID) return 1;
+  if (sg_transfer_budget(32, 1024, 0.5, 1.0) != 15872) return 2;              /* Eq. 2: M (L-1) T_p / T_t */
+  if (sg_transfer_budget(32, 1024, 1e-9, 1.0) != 2048) return 3;              /* clipped to 2M */
+  if (sg_speculative_delivered(32, 1024, 2048, 0.10, 10) != 32768) return 4;  /* 10 % per iteration */
+  if (strcmp(sg_strerror(SG_OK), "ok") != 0) return 5;
+  printf("c caller ok\n");
+  return 0;
+}
+''')
+    exe = tmp_path / "caller"
+    libdir = os.path.dirname(sg.LIB_PATH)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe),
+                    "-L", libdir, "-lsmartgen", "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout
+    assert "c caller ok" in out
