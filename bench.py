@@ -352,7 +352,8 @@ def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (
         nbytes = Hkv * (2 * (Ktot + NL) * d * 2 + NL * 4) + 2 * B * Hq * d * 2
         gbs = nbytes / us / 1e3
         out.append({"batch": B, "sel": sel, "rho": rho, "n_sel": Ktot // B, "n_loc": NL // B, "us_per_call": us,
-                    "bytes_per_call": nbytes, "achieved_gbs": gbs, "frac_of_copy_peak": gbs / peaks["hbm_gbs"],
+                    "bytes_per_call": nbytes, "l2": "larger than L2" if nbytes > 126e6 else "warm L2 (same buffers every call)",
+                    "achieved_gbs": gbs, "frac_of_copy_peak": gbs / peaks["hbm_gbs"],
                     "tokens_per_s": B / (us * 1e-6)})
         del k, v, pk, pv
         torch.cuda.empty_cache()
@@ -655,10 +656,27 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode-sweep", action="store_true", help="skip the extra decode-only points (c2 only)")
+    ap.add_argument("--decode-sweep-grid", action="store_true",
+                    help="only the decode-heavy sweep: sg_sparse_decode_attn alone on batch {1, 8, 32, 128} x required "
+                         "fraction {5, 20, 100 %} x index-addressed share {0, 25, 50 %}; prints one JSON line and exits")
     ap.add_argument("--no-extras", action="store_true",
                     help="only the timed step: skip the decode sweep, the timings of the other entry points, the "
                          "layer-by-layer prefill and the pipelined e2e (for profiling the step itself)")
     args = ap.parse_args()
+    if args.decode_sweep_grid:
+        import torch
+        from paper_2607_28150_b200 import build as _build
+        if not os.path.exists(_build.LIB):
+            _build.build()
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+        dev = torch.device("cuda", 0)
+        torch.cuda.set_device(dev)
+        points = tuple((b, sel, rho) for b in (1, 8, 32, 128) for sel in (0.05, 0.2, 1.0) for rho in (0.0, 0.25, 0.5))
+        peaks = load_peaks()
+        print(json.dumps({"decode_sweep_grid": decode_sweep_points(dev, peaks, points), "peak_gbs": peaks["hbm_gbs"],
+                          "peak_source": peaks["source"], "calls_per_graph": 16}))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
