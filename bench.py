@@ -380,6 +380,8 @@ def run_ours(args):
     L, B, Hq, Hkv, d, W = cfg.num_layers, cfg.batch, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.window
     T = cfg.total_tokens
     nsteps_dec = args.decode_steps if args.decode_steps is not None else cfg.decode_steps
+    if args.decode_steps is None and args.workload == "c5":
+        nsteps_dec = 16        # a single call per graph would measure the graph launch, not the kernel
     nloc = cfg.n_local()
     cu_nloc_h = np.concatenate([[0], np.cumsum(nloc)]).astype(np.int32)
     NL = int(cu_nloc_h[-1])
