@@ -8,8 +8,8 @@ sg_select_topk and sg_pack_kv over all layers (one call each), then the workload
 (one sg_sparse_decode_attn call per layer per step, replayed from a CUDA graph).  The default
 workload is the Llama-3-8B-shaped cache (32 layers, 8192-token prompt, 10 % budget, 64 decode
 steps).  Rank 0 prints ONE JSON line:
-  value                 (select + pack algorithmic bytes) / device time from the start of the selection kernel to the end of
-                        the packing kernel launched right behind it, inputs resident in HBM
+  value                 (select + pack algorithmic bytes) / device time of the sg_select_pack_kv call (selection and gather in
+                        one kernel on this workload), inputs resident in HBM; stage_ms.select / .pack: the two separate calls
   decode_tokens_per_s   batch * decode steps / decode-stage device time;  stage_ms: every stage of a step
   e2e                   the same step with host buffers (pinned H2D of caches and queries, D2H of the payload and outputs)
   roofline / rooflines  per-kernel achieved bytes/s (or flop/s) against the measured copy / bf16 peaks
@@ -460,19 +460,21 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     def step(e2e: bool, ev, split: bool = False):
-        """One pass of the path.  `ev` is a list of 7 events bracketing: h2d | score | select, pack | d2h | decode.
-        The selection and the packing kernel run back to back, as a caller launches them; only a `split` pass puts an
-        event between the two (ev[3]), which costs 2-3 us of idle device time and is used for the per-kernel times."""
+        """One pass of the path.  `ev` is a list of 7 events bracketing: h2d | score | select + pack | d2h | decode.
+        Selection and packing are one library call (sg_select_pack_kv: one fused kernel on this workload); a `split`
+        pass makes the two separate calls with an event between them (ev[3]) and gives the per-kernel times."""
         ev[0].record(stream)
         if e2e:
             d_q.copy_(h_q, non_blocking=True); d_k.copy_(h_k, non_blocking=True); d_v.copy_(h_v, non_blocking=True)
         ev[1].record(stream)
         hp.score(d_q, d_k)
         ev[2].record(stream)
-        hp.select()
         if split:
+            hp.select()
             ev[3].record(stream)
-        hp.pack(d_k, d_v)
+            hp.pack(d_k, d_v)
+        else:
+            hp.select_pack(d_k, d_v)
         ev[4].record(stream)
         if e2e:
             h_pk.copy_(hp.packed_k, non_blocking=True); h_pv.copy_(hp.packed_v, non_blocking=True)
@@ -505,6 +507,8 @@ def run_ours(args):
         stage = {n: sum(e[a].elapsed_time(e[b]) for e in evs) / steps for n, (a, b) in spans.items()}
         # per-kernel times of the two kernels inside the span, from passes with an event between them (not part of total_ms)
         sevs = [mk() for _ in range(steps)]
+        for _ in range(min(warmup, 2)):
+            step(e2e, mk(), split=True)
         for i in range(steps):
             step(e2e, sevs[i], split=True)
         torch.cuda.synchronize()
@@ -585,7 +589,10 @@ def run_ours(args):
         "score": hbm("score", work["score"]["bytes"], st["score"], 1),
         "select": hbm("select", work["select"]["bytes"], st["select"], 1),
         "pack": hbm("pack", work["pack"]["bytes"], st["pack"], 1),
+        "select_pack": hbm("select_pack", work["select"]["bytes"] + work["pack"]["bytes"], st["select_pack"], 1),
     }
+    for n in ("select", "pack"):
+        roofs[n]["launches_per_step"] = 0       # timed in the split passes; the step itself runs the fused kernel
     roofs["score"]["tensor_tflops"] = work["score"]["flops"] / (st["score"] * 1e-3) / 1e12
     roofs["score"]["tensor_frac_of_sustained"] = roofs["score"]["tensor_tflops"] / tc_peak
     roofs["select"]["rows"] = L * B * Hkv
@@ -640,7 +647,7 @@ def run_ours(args):
         "stage_ms": st,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
-        "gpu_launches": args.steps * (3 + ncalls_dec),
+        "gpu_launches": args.steps * (2 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
         "decode_sweep": sweep, "next_rows": next_rows, "prefill_layerwise": layerwise,
         "e2e_pipelined": None if ms_pipe is None else {

@@ -122,6 +122,19 @@ sg_status sg_pack_kv(const sg_shape* shape, const void* k_cache, const void* v_c
                      void* packed_v, int32_t* dev_status, void* stream);
 
 /*
+ * sg_select_pack_kv -- sg_select_topk followed by sg_pack_kv in one call: the prefill node selects the
+ * required entries and gathers them for sending (Section 4.2).  Writes exactly what the two calls write:
+ * sel_idx (the KV index, which travels with the payload) and packed_k / packed_v, with the same device status
+ * bits.  When every row has at most 32768 tokens and there are at least as many (layer, sequence, KV head)
+ * rows as SMs, one kernel does both: the CTA that selected a row gathers that row's K/V, so the latency-bound
+ * selection of some rows overlaps the bandwidth-bound gather of others.  Otherwise the two kernels are launched
+ * back to back.  Arguments as in sg_select_topk and sg_pack_kv; no workspace; asynchronous on `stream`.
+ */
+sg_status sg_select_pack_kv(const sg_shape* shape, const float* importance, const int32_t* cu_k,
+                            int32_t total_sel, const void* k_cache, const void* v_cache, int32_t* sel_idx,
+                            void* packed_k, void* packed_v, int32_t* dev_status, void* stream);
+
+/*
  * sg_sparse_decode_attn -- one decode step of attention over a two-source KV list.
  *
  * Defines: two-lane KV fetching (Section 4.2): the entries a head needs arrive partly as

@@ -21,7 +21,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
-            "sg_score_static", "sg_select_threshold", "sg_pack_kv_counted", "sg_sparse_decode_attn_counted", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
+            "sg_score_static", "sg_select_pack_kv", "sg_select_threshold", "sg_pack_kv_counted", "sg_sparse_decode_attn_counted", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
             "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -74,6 +74,8 @@ _lib.sg_speculative_delivered.restype = ctypes.c_int64
 _lib.sg_speculative_delivered.argtypes = [_i32, _i32, ctypes.c_int64, ctypes.c_double, _i32]
 _lib.sg_proactive_mask.restype = ctypes.c_int
 _lib.sg_proactive_mask.argtypes = [_sp, _i32, _i32, _vp, _i32, _vp, _vp]
+_lib.sg_select_pack_kv.restype = ctypes.c_int
+_lib.sg_select_pack_kv.argtypes = [_sp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_pack_kv_counted.restype = ctypes.c_int
 _lib.sg_pack_kv_counted.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.sg_sparse_decode_attn_counted.restype = ctypes.c_int
@@ -288,6 +290,20 @@ def sg_select_threshold(shape: Shape, scores: torch.Tensor, alpha: float, cu_cap
                                   _ptr(sel_count), _ptr(dev_status), _stream(stream))
     if rc:
         raise SmartGenError(rc, "sg_select_threshold")
+
+
+def sg_select_pack_kv(shape: Shape, importance: torch.Tensor, cu_k: torch.Tensor, total_sel: int, k_cache: torch.Tensor,
+                      v_cache: torch.Tensor, sel_idx: torch.Tensor, packed_k: torch.Tensor, packed_v: torch.Tensor,
+                      dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """sg_select_topk then sg_pack_kv in one call (one fused kernel where that pays); same outputs as the two calls."""
+    _check(importance, torch.float32, "importance"); _check(cu_k, torch.int32, "cu_k")
+    _check(k_cache, _BF16, "k_cache"); _check(v_cache, _BF16, "v_cache"); _check(sel_idx, torch.int32, "sel_idx", total_sel == 0)
+    _check(packed_k, _BF16, "packed_k", total_sel == 0); _check(packed_v, _BF16, "packed_v", total_sel == 0)
+    _check(dev_status, torch.int32, "dev_status", True)
+    rc = _lib.sg_select_pack_kv(ctypes.byref(shape), _ptr(importance), _ptr(cu_k), total_sel, _ptr(k_cache), _ptr(v_cache),
+                                _ptr(sel_idx), _ptr(packed_k), _ptr(packed_v), _ptr(dev_status), _stream(stream))
+    if rc:
+        raise SmartGenError(rc, "sg_select_pack_kv")
 
 
 def sg_pack_kv_counted(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tensor, sel_idx: torch.Tensor,

@@ -67,10 +67,15 @@ class HotPath:
                       self.status, stream)
         return self.packed_k, self.packed_v
 
+    def select_pack(self, k_cache: torch.Tensor, v_cache: torch.Tensor, stream=None):
+        """select() then pack() as one library call (one fused kernel where the library finds that it pays)."""
+        sg.sg_select_pack_kv(self.shape, self.importance, self.cu_k, self.K_tot, k_cache, v_cache, self.sel_idx,
+                             self.packed_k, self.packed_v, self.status, stream)
+        return self.packed_k, self.packed_v
+
     def prefill(self, q_win, k_cache, v_cache, stream=None):
         self.score(q_win, k_cache, stream)
-        self.select(stream)
-        return self.pack(k_cache, v_cache, stream)
+        return self.select_pack(k_cache, v_cache, stream)
 
     def prefill_layer(self, layer: int, q_win: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
                       stream=None, aux_stream=None):

@@ -88,6 +88,22 @@ def pack_kv(k_cache, v_cache, cu, sel_idx, cu_k, expect_status=0):
     return a, b
 
 
+def select_pack_kv(importance, k_cache, v_cache, cu, cu_k, expect_status=0):
+    L, T, Hkv, d = k_cache.shape
+    shp = shape_of(L, Hkv, Hkv, d, 1, cu)
+    cu_k = np.asarray(cu_k, dtype=np.int32)
+    Ktot = int(cu_k[-1])
+    sel = Guarded((L, Hkv, Ktot), torch.int32, -99)
+    pk = Guarded((L, Ktot * Hkv, d), torch.int16, 0x5555)
+    pv = Guarded((L, Ktot * Hkv, d), torch.int16, 0x5555)
+    st = status_word()
+    sg.sg_select_pack_kv(shp, dev(np.asarray(importance, np.float32)), dev(cu_k), Ktot, dev(k_cache), dev(v_cache),
+                         sel.view, pk.view, pv.view, st)
+    s_, a, b = sel.numpy(), pk.numpy(), pv.numpy()
+    assert read_status(st) == expect_status
+    return s_, a, b
+
+
 def sparse_decode_attn(q, packed_k, packed_v, cu_k, local_k, local_v, cu, local_idx, cu_nloc, softmax_scale=0.0,
                        expect_status=0):
     B, Hq, d = q.shape

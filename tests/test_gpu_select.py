@@ -61,3 +61,24 @@ def test_select_budget_above_length_is_flagged():
     x = np.arange(8, dtype=np.float32)[None, None]
     got = gpu_ops.select_topk(x, cu_of((8,)), cu_of((10,)), expect_status=1 << sg.SG_ERR_INVALID)
     assert got[0, 0].tolist() == list(range(8)) + [-1, -1]
+
+
+def test_select_narrow_clustered_and_wide_key_ranges():
+    """Rows whose values span a few ulps, rows with half of the values inside a 4096-ulp cluster that holds the threshold
+    (many keys stay in the interval after two narrowing passes), and rows spread over the whole float range."""
+    rng = np.random.default_rng(7)
+    n = 8192
+    one = np.float32(1.0).view(np.uint32)
+    narrow = (one + rng.integers(0, 40, size=(1, 4, n)).astype(np.uint32)).view(np.float32)
+    check(narrow, (n,), (820,))
+    bits = (np.uint32(0x10000000) + rng.integers(0, 1 << 29, size=(1, 4, n)).astype(np.uint32))
+    cluster = rng.random((1, 4, n)) < 0.5
+    bits[cluster] = one + rng.integers(0, 4096, size=int(cluster.sum())).astype(np.uint32)
+    clustered = bits.view(np.float32)
+    check(clustered, (n,), (820,))
+    check(np.ascontiguousarray(clustered[:, :, :8190]), (5001, 3189), (4000, 7))     # unaligned second row
+    wide = (rng.standard_normal((2, 4, n)) * 10.0 ** rng.uniform(-35, 35, size=(2, 4, n))).astype(np.float32)
+    wide[:, :, ::97] = np.float32(np.inf)
+    wide[:, :, 5::101] = -np.float32(np.inf)
+    check(wide, (n,), (1000,))
+    check(wide, (4096, 4096), (4000, 2))
