@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelPa
 // selection another streams rows: the two phases overlap across CTAs without any inter-CTA wait.
 constexpr int kPackUnroll = 4;
 constexpr int kFinishMax = 64;                         // interval populations up to this are finished by direct ranking
-constexpr int64_t kFuseMinRows = 148;
+constexpr int64_t kFuseMinRows = kNumSMs;               // fewer rows than SMs cannot fill the machine with their gathers
 constexpr int kRegBins = 2048;
 constexpr int kRegCopies = 2;
 
