@@ -81,6 +81,19 @@ int main(void) {
       }
     }
   }
+  {
+    /* the one-call form writes what the two calls wrote */
+    int* d_sel2; unsigned short *d_pk2, *d_pv2;
+    int* sel2 = (int*)malloc(n_sel * 4);
+    unsigned short* pk2 = (unsigned short*)malloc(n_pk * 2); unsigned short* pv2 = (unsigned short*)malloc(n_pk * 2);
+    CK(cudaMalloc((void**)&d_sel2, n_sel * 4)); CK(cudaMalloc((void**)&d_pk2, n_pk * 2)); CK(cudaMalloc((void**)&d_pv2, n_pk * 2));
+    if (sg_select_pack_kv(&s, d_imp, d_cuk, KT, d_k, d_v, d_sel2, d_pk2, d_pv2, d_status, NULL) != SG_OK) return 40;
+    CK(cudaDeviceSynchronize());
+    CK(cudaMemcpy(sel2, d_sel2, n_sel * 4, cudaMemcpyDeviceToHost)); CK(cudaMemcpy(status, d_status, 16, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(pk2, d_pk2, n_pk * 2, cudaMemcpyDeviceToHost)); CK(cudaMemcpy(pv2, d_pv2, n_pk * 2, cudaMemcpyDeviceToHost));
+    if (status[0] != 0) return 41;
+    if (memcmp(sel2, sel, n_sel * 4) != 0 || memcmp(pk2, pk, n_pk * 2) != 0 || memcmp(pv2, pv, n_pk * 2) != 0) return 42;
+  }
   printf("c caller on the gpu ok\n");
   return 0;
 }
