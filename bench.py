@@ -305,6 +305,41 @@ def layerwise_prefill_timing(dev, hp, d_q, d_k, d_v, reps=5):
             "note": "3 kernels + 1 counter memset per layer; compare with score+select+pack of the all-layer calls in stage_ms"}
 
 
+def full_first_two_timing(dev, cfg, d_q, d_k, d_v, reps=5):
+    """The prefill side under the budget policy of Eq. 1 / Eq. 2's clip: layers 0 and 1 are transferred whole
+    (k_b = N_b, the selection degenerates to the identity list), the other layers get the workload's budget.
+    Two call groups replayed from one CUDA graph; device ms and the payload it produces."""
+    import torch
+    from paper_2607_28150_b200.pipeline import HotPath
+    L = cfg.num_layers
+    if L <= 2:
+        return None
+    args = (cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.window, cfg.seqlens)
+    first = HotPath(2, *args, list(cfg.seqlens), device=dev)
+    rest = HotPath(L - 2, *args, cfg.budgets(), device=dev)
+
+    def run():
+        first.select_pack(d_k[:2], d_v[:2])
+        rest.prefill(d_q[2:], d_k[2:], d_v[2:])
+
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        run(); side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            run()
+        g.replay(); side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for _ in range(reps):
+            g.replay()
+        e1.record(side); side.synchronize()
+    status = first.read_status() | rest.read_status()
+    payload = 2 * (first.packed_k.numel() + rest.packed_k.numel()) * 2 + (first.sel_idx.numel() + rest.sel_idx.numel()) * 4
+    return {"ms_prefill": e0.elapsed_time(e1) / reps, "payload_mb": payload / 1e6, "dev_status": status,
+            "note": "layers 0-1 with k_b = N_b (whole layers), layers 2..%d with the workload's budget; score + select + pack" % (L - 1)}
+
+
 def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (128, 1.0, 0.5)), calls=16):
     """sg_sparse_decode_attn alone on points of the decode-heavy sweep (B sequences of 4096 tokens, `sel` of the
     prompt required, `rho` of that index-addressed): the sizes at which the kernel can reach the HBM roofline.
@@ -629,6 +664,7 @@ def run_ours(args):
     kv_mib = (h_k.numel() + h_v.numel()) * 2 / 2**20
     next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 and not args.no_extras else None
     layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
+    first_two = full_first_two_timing(dev, cfg, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
     sweep = None
     if args.workload == "c2" and not args.no_decode_sweep and not args.no_extras and world == 1:
         del d_k, d_v, h_k, h_v
@@ -650,7 +686,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (2 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "decode_sweep": sweep, "next_rows": next_rows, "prefill_layerwise": layerwise,
+        "decode_sweep": sweep, "next_rows": next_rows, "prefill_layerwise": layerwise, "prefill_full_first_two": first_two,
         "e2e_pipelined": None if ms_pipe is None else {
             "ms_prefill": ms_pipe, "value": sp_bytes / (ms_pipe * 1e-3) / 1e9, "unit": UNIT,
             "note": "host buffers, layer by layer on three streams (copy in | score, select, pack | copy out); "
