@@ -81,3 +81,28 @@ def test_fused_oversized_budget_sets_both_bits_and_zero_rows():
     # the first sequence is a normal selection
     want = oracle.select_topk(np.ascontiguousarray(imp[:, :, :100]), cu_of((100,)), cu_of((10,)))
     assert np.array_equal(sel[:, :, :10], want)
+
+
+def test_fused_strided_cache_view():
+    """The fused kernel gathers through the cache strides of the shape: a cache whose token stride is wider than
+    H_kv * d (a slice of a larger allocation), 160 rows so that the one-kernel route is taken."""
+    import torch
+    import gpu_ops
+    import paper_2607_28150_b200.binding as sg
+    lens, ks, L, Hkv, d = (200, 77), (33, 8), 10, 8, 128
+    imp, k, v, cu, ck = case(8, lens, ks, L, Hkv, d)
+    T, pad, Ktot = int(cu[-1]), 2, int(ck[-1])
+    kbig = np.zeros((L, T, Hkv + pad, d), dtype=np.uint16); kbig[:, :, :Hkv] = k
+    vbig = np.zeros_like(kbig); vbig[:, :, :Hkv] = v
+    shp = gpu_ops.shape_of(L, Hkv, Hkv, d, 1, cu, layer_stride=T * (Hkv + pad) * d, token_stride=(Hkv + pad) * d)
+    sel = torch.full((L, Hkv, Ktot), -99, dtype=torch.int32, device="cuda")
+    pk = torch.zeros((L, Ktot * Hkv, d), dtype=torch.int16, device="cuda")
+    pv = torch.zeros_like(pk)
+    st = gpu_ops.status_word()
+    sg.sg_select_pack_kv(shp, gpu_ops.dev(imp), gpu_ops.dev(ck), Ktot, gpu_ops.dev(kbig), gpu_ops.dev(vbig), sel, pk, pv, st)
+    assert gpu_ops.read_status(st) == 0
+    want_sel = oracle.select_topk(imp, cu, ck)
+    want_k, want_v = oracle.pack_kv(k, v, cu, want_sel, ck)
+    assert np.array_equal(sel.cpu().numpy(), want_sel)
+    assert np.array_equal(pk.cpu().numpy().view(np.uint16), want_k)
+    assert np.array_equal(pv.cpu().numpy().view(np.uint16), want_v)
