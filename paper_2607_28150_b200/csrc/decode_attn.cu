@@ -208,6 +208,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
 
   // Everything above reads only the KV sources, the index lists and the prefix arrays, which are stable
   // inputs of a decode step; q (and the outputs) are ordered after all earlier work in the stream.
+  // Only an L2 prefetch of the query rows is issued early: L2 is where writes of earlier kernels land, so the
+  // loads behind the wait see current data, and find it on chip when nobody rewrote it in between.
+  if (warp == 0 && lane * 64 < p.G * D)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.q + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D + lane * 64));
   pdl_wait();
   // Q fragments (A operand, 16 x D, rows >= G are zero).
   const int r_lo = lane >> 2, r_hi = r_lo + 8;
