@@ -463,7 +463,10 @@ sg_status select_launch(const sg_shape* shape, SelParams& p, bool fuse, void* st
     else if (pd == 64) SG_LAUNCH_SELECT_REG_PD(E, T, 64); \
     else SG_LAUNCH_SELECT_REG_PD(E, T, 0);                \
   } while (0)
-  if (shape->max_seqlen <= 4096) {
+  if (rows < kNumSMs && !fuse && shape->max_seqlen <= 8192 && shape->max_seqlen > 4096) {
+    // fewer rows than SMs: one CTA per SM anyway, so twice the threads per row (half the keys each) shorten the chains
+    SG_LAUNCH_SELECT_REG_PD(8, 1024, 0);
+  } else if (shape->max_seqlen <= 4096) {
     SG_LAUNCH_SELECT_REG(8, 512);
   } else if (shape->max_seqlen <= 8192) {
     SG_LAUNCH_SELECT_REG(16, 512);
