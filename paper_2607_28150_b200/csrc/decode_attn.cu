@@ -89,6 +89,11 @@ __device__ __forceinline__ void st_dsmem_f32(float* local_ptr, uint32_t cta_rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
   asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(remote), "f"(v) : "memory");
 }
+__device__ __forceinline__ void st_dsmem_f32x2(float* local_ptr, uint32_t cta_rank, float a, float b) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(remote), "f"(a), "f"(b) : "memory");
+}
 // Programmatic dependent launch: let the next kernel in the stream start its prologue now, and wait
 // for the previous kernel's memory before touching anything it may have written.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -338,8 +343,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   __syncthreads();
 
   // merge the warps through shared memory (the rings are free now)
-  float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][D]
-  float* sm_m = sm_o + kDecWarps * 16 * D;                    // [kDecWarps][16]
+  constexpr int kOStride = D + 8;                             // row stride of the partials: the rows of a store land in different banks
+  float* sm_o = reinterpret_cast<float*>(smem_raw);           // [kDecWarps][16][kOStride]
+  float* sm_m = sm_o + kDecWarps * 16 * kOStride;             // [kDecWarps][16]
   float* sm_l = sm_m + kDecWarps * 16;
   const bool w_lo = r_lo < p.G, w_hi = kHi && r_hi < p.G;      // rows >= G are padding and never read
   if ((lane & 3) == 0) {
@@ -349,9 +355,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
 #pragma unroll
   for (int i = 0; i < D / 8; ++i) {
     const int col = i * 8 + 2 * (lane & 3);
-    float* dst = sm_o + (warp * 16 + r_lo) * D + col;
+    float* dst = sm_o + (warp * 16 + r_lo) * kOStride + col;
     if (w_lo) *reinterpret_cast<float2*>(dst) = make_float2(o_acc[i][0], o_acc[i][1]);
-    if (w_hi) *reinterpret_cast<float2*>(dst + 8 * D) = make_float2(o_acc[i][2], o_acc[i][3]);
+    if (w_hi) *reinterpret_cast<float2*>(dst + 8 * kOStride) = make_float2(o_acc[i][2], o_acc[i][3]);
   }
   __syncthreads();
   // CTA-level partial of every output; with a cluster, each rank owns a slice of the G*d outputs and
@@ -361,27 +367,31 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
   float* lsep = p.lse ? p.lse + (int64_t)b * p.Hq + (int64_t)g * p.G : nullptr;
   if (cs > 1) cluster_wait();                                  // every CTA of the cluster has started
-  for (int e = tid; e < p.G * D; e += kDecThreads) {
+  // two neighbouring outputs per thread (same row, same owner: D and the owners' slices are even)
+  for (int e = 2 * tid; e < p.G * D; e += 2 * kDecThreads) {
     const int r = e / D, col = e - r * D;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, sm_m[w * 16 + r]);
     const float Mu = M == -INFINITY ? 0.f : M;
-    float L = 0.f, O = 0.f;
+    float L = 0.f, O0 = 0.f, O1 = 0.f;
 #pragma unroll
     for (int w = 0; w < kDecWarps; ++w) {
       const float f = exp2f(sm_m[w * 16 + r] - Mu);
+      const float2 o = *reinterpret_cast<const float2*>(sm_o + (w * 16 + r) * kOStride + col);
       L += sm_l[w * 16 + r] * f;
-      O += sm_o[(w * 16 + r) * D + col] * f;
+      O0 += o.x * f;
+      O1 += o.y * f;
     }
     if (cs == 1) {
-      outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+      *reinterpret_cast<__nv_bfloat162*>(outp + e) = __floats2bfloat162_rn(L > 0.f ? O0 / L : 0.f, L > 0.f ? O1 / L : 0.f);
       if (lsep && col == 0) lsep[r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     } else {
       const int owner = e / per;
-      st_dsmem_f32(rx_o + c * per + (e - owner * per), owner, O);
-      if (col == 0) {
-        for (int j = 0; j < cs; ++j) { st_dsmem_f32(rx_m + c * 16 + r, j, M); st_dsmem_f32(rx_l + c * 16 + r, j, L); }
+      st_dsmem_f32x2(rx_o + c * per + (e - owner * per), owner, O0, O1);
+      if ((col >> 1) < cs) {                                  // the row's (M, L) goes to every rank: one thread per rank
+        st_dsmem_f32(rx_m + c * 16 + r, col >> 1, M);
+        st_dsmem_f32(rx_l + c * 16 + r, col >> 1, L);
       }
     }
   }
