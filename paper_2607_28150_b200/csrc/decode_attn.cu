@@ -77,22 +77,34 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
-}
-__device__ __forceinline__ void cluster_arrive_relaxed() {
-  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n" ::: "memory");
-}
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory"); }
-__device__ __forceinline__ void st_dsmem_f32(float* local_ptr, uint32_t cta_rank, float v) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
-  asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(remote), "f"(v) : "memory");
+// Remote stores that report their bytes to an mbarrier of the destination CTA: the owner of an output slice waits on
+// its own barrier for everybody's partials instead of the whole cluster meeting at a barrier.
+__device__ __forceinline__ void st_async_f32(float* local_ptr, uint64_t* local_bar, uint32_t cta_rank, float v) {
+  uint32_t raddr, rbar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(raddr) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(rbar) : "r"(smem_u32(local_bar)), "r"(cta_rank));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];\n" ::"r"(raddr), "f"(v), "r"(rbar) : "memory");
 }
-__device__ __forceinline__ void st_dsmem_f32x2(float* local_ptr, uint32_t cta_rank, float a, float b) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(remote), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ void st_async_f32x2(float* local_ptr, uint64_t* local_bar, uint32_t cta_rank, float a, float b) {
+  uint32_t raddr, rbar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(raddr) : "r"(smem_u32(local_ptr)), "r"(cta_rank));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(rbar) : "r"(smem_u32(local_bar)), "r"(cta_rank));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n" ::"r"(raddr), "f"(a), "f"(b), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+}
+// Bounded wait for phase 0 of an mbarrier whose bytes come from other CTAs of the cluster; false when it gave up.
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar) {
+  const uint32_t addr = smem_u32(bar);
+  for (int it = 0; it < (1 << 16); ++it) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                 : "=r"(done) : "r"(addr) : "memory");
+    if (done) return true;
+  }
+  return false;
 }
 // Programmatic dependent launch: let the next kernel in the stream start its prologue now, and wait
 // for the previous kernel's memory before touching anything it may have written.
@@ -118,11 +130,25 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   float* rx_m = reinterpret_cast<float*>(s_mask + kDecWarps * kBuf);
   float* rx_l = rx_m + 8 * 16;
   float* rx_o = rx_l + 8 * 16;
+  uint64_t* rx_bar = reinterpret_cast<uint64_t*>(rx_o + 16 * D);   // counts the bytes of the partials pushed into the three arrays
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.y;
   pdl_launch_dependents();
-  if (p.csize > 1) cluster_arrive_relaxed();                   // "this CTA runs": awaited before the first remote store
+  if (p.csize > 1) {
+    if (tid == 0) {
+      // every rank sends this CTA its partial of the slice owned here and its (M, L) of the G rows
+      const int per0 = (p.G * D + p.csize - 1) / p.csize;
+      const int c_rank = blockIdx.x % p.csize;
+      const int own = max(0, min(p.G * D, (c_rank + 1) * per0) - c_rank * per0);
+      const uint32_t bytes = (uint32_t)p.csize * (uint32_t)(own + 2 * p.G) * 4u;
+      const uint32_t bar = smem_u32(rx_bar);
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" ::"r"(bar) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+    }
+    cluster_arrive_release();                                  // "this CTA runs, its barrier is set up": awaited before the first remote store
+  }
   const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
   const int kb = p.cu_k[b + 1] - p.cu_k[b];                    // packed rows per KV head (the slot size in the buffer)
@@ -388,16 +414,21 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       if (lsep && col == 0) lsep[r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     } else {
       const int owner = e / per;
-      st_dsmem_f32x2(rx_o + c * per + (e - owner * per), owner, O0, O1);
+      st_async_f32x2(rx_o + c * per + (e - owner * per), rx_bar, owner, O0, O1);
       if ((col >> 1) < cs) {                                  // the row's (M, L) goes to every rank: one thread per rank
-        st_dsmem_f32(rx_m + c * 16 + r, col >> 1, M);
-        st_dsmem_f32(rx_l + c * 16 + r, col >> 1, L);
+        st_async_f32(rx_m + c * 16 + r, rx_bar, col >> 1, M);
+        st_async_f32(rx_l + c * 16 + r, rx_bar, col >> 1, L);
       }
     }
   }
   if (cs > 1) {
-    cluster_sync_all();                                       // release the pushes, acquire everyone else's
+    // Only the threads that merge wait, and only for the bytes addressed to this CTA.  Once they are all here nobody
+    // writes into this CTA's shared memory any more, so it may finish without meeting the others again.
     const int e_beg = c * per, e_end = min(p.G * D, e_beg + per);
+    if ((e_beg + tid < e_end || tid == 0) && !mbar_wait_cluster_bounded(rx_bar)) {   // thread 0 keeps the CTA alive for its senders in any case
+      raise(p.dev_status, SG_ERR_TIMEOUT);
+      return;
+    }
     for (int e = e_beg + tid; e < e_end; e += kDecThreads) {
       const int r = e / D, col = e - r * D;
       float mj[8], lj[8], oj[8];
@@ -422,13 +453,12 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       outp[e] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
       if (lsep && col == 0) lsep[r] = L > 0.f ? (M + log2f(L)) * kLn2 : -INFINITY;
     }
-    // no trailing barrier: after the one above nobody touches another CTA's shared memory
   }
 }
 
 template <int D, int kDecWarps, int kBuf>
 constexpr int decode_smem_bytes() {
-  return kDecWarps * kBuf * 2 * kSlice * D * 2 + kDecWarps * kBuf * 4 + (2 * 8 * 16 + 16 * D) * 4;   // rings, masks, receive area
+  return kDecWarps * kBuf * 2 * kSlice * D * 2 + kDecWarps * kBuf * 4 + (2 * 8 * 16 + 16 * D) * 4 + 16;   // rings, masks, receive area, its barrier
 }
 
 }  // namespace
