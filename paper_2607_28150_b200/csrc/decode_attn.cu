@@ -476,9 +476,14 @@ void decode_plan(const sg_shape* shape, int32_t total_sel, int32_t total_loc, in
   const int64_t avg_tokens = ((int64_t)total_sel + total_loc) / shape->batch;
   int W = 4, cs = 1;
   if (pairs <= kNumSMs) {
-    W = 8;
+    // largest cluster whose CTAs are all resident at once; clusters of eight one-CTA-per-SM CTAs must also leave half
+    // of the SMs to the next call, whose clusters cannot be placed otherwise while this call drains (2x slower)
     int fit = 1;
     while (fit < 8 && pairs * fit * 2 <= kNumSMs) fit *= 2;
+    const int fit8 = (fit == 8 && pairs * 16 > kNumSMs) ? 4 : fit;
+    // short lists: four warps per CTA already give every warp at most ~1.75 slices, and the merge is half as wide
+    W = 4 * avg_tokens <= 7 * 4 * kSlice * fit ? 4 : 8;
+    if (W == 8) fit = fit8;
     int work = 1;
     while (work < 8 && (int64_t)work * W * kSlice < avg_tokens) work *= 2;
     cs = fit < work ? fit : work;
