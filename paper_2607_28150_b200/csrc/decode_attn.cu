@@ -98,12 +98,13 @@ __device__ __forceinline__ void cluster_arrive_release() {
 // Bounded wait for phase 0 of an mbarrier whose bytes come from other CTAs of the cluster; false when it gave up.
 __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint64_t* bar) {
   const uint32_t addr = smem_u32(bar);
-  for (int it = 0; it < (1 << 16); ++it) {
+  const long long t0 = clock64();
+  do {                                                      // the senders run concurrently (same cluster): microseconds; the limit is ~0.5 s
     uint32_t done;
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                  : "=r"(done) : "r"(addr) : "memory");
     if (done) return true;
-  }
+  } while (clock64() - t0 < 1000000000LL);
   return false;
 }
 // Programmatic dependent launch: let the next kernel in the stream start its prologue now, and wait
