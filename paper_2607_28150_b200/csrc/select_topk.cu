@@ -187,7 +187,8 @@ constexpr int64_t kFuseMinRows = kNumSMs;               // fewer rows than SMs c
 constexpr int kRegBins = 2048;
 constexpr int kRegCopies = 2;
 
-// Block-wide exclusive prefix sum of one value per thread (T threads); `wsum` holds 2*T/32 words.
+// Block-wide exclusive prefix sum of one value per thread (T threads); `wsum` holds T/32 words.  One barrier: every
+// warp adds up the totals of the warps before it by itself.  The caller keeps a barrier between two calls.
 template <int T>
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* wsum, int lane, int warp) {
   uint32_t inc = v;
@@ -198,18 +199,8 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
   }
   if (lane == 31) wsum[warp] = inc;
   __syncthreads();
-  if (warp == 0) {
-    const uint32_t w = lane < T / 32 ? wsum[lane] : 0u;
-    uint32_t wi = w;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t u = __shfl_up_sync(0xffffffffu, wi, off);
-      if (lane >= off) wi += u;
-    }
-    if (lane < T / 32) wsum[T / 32 + lane] = wi - w;
-  }
-  __syncthreads();
-  return wsum[T / 32 + warp] + inc - v;
+  const uint32_t before = __reduce_add_sync(0xffffffffu, (lane < T / 32 && lane < warp) ? wsum[lane] : 0u);
+  return before + inc - v;
 }
 
 template <int E, int T, int PD>
