@@ -278,8 +278,11 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
     constexpr int wrow = 0;
 
     // S = Q K^T for 16 tokens (two n8 tiles)
+    // (even and odd k-steps accumulate separately: two dependent chains of half the length; a warp has only one or two
+    // slices at small batch, so the length of this chain is what it waits for)
     float s_acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     {
+      float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
       const int mi = lane >> 3;
       const int row = wrow + (mi >> 1) * 8 + (lane & 7);
 #pragma unroll
@@ -287,8 +290,13 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
         const int chunk = kk * 2 + (mi & 1);
         uint32_t kf[4];
         ldmatrix_x4(kf, k_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
-        mma_bf16(s_acc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[0], kf[1]);
-        mma_bf16(s_acc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[2], kf[3]);
+        mma_bf16((kk & 1) ? s_odd[0] : s_acc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[0], kf[1]);
+        mma_bf16((kk & 1) ? s_odd[1] : s_acc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[2], kf[3]);
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s_acc[j][e] += s_odd[j][e];
       }
     }
     // online softmax in base 2; mask padding and skipped indices
@@ -336,14 +344,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
         pa[2 * j + 1] = 0u;
       }
     }
-    sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1);
-    sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
+    // the four lanes of a row keep their own part of the row sum (the rescale factor is the same for all four);
+    // the parts are added up once, after the last slice
     l_lo = l_lo * al_lo + sum_lo;
-    if (kHi) {
-      sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1);
-      sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
-      l_hi = l_hi * al_hi + sum_hi;
-    }
+    if (kHi) l_hi = l_hi * al_hi + sum_hi;
     const bool rescale = kHi ? (al_lo != 1.f || al_hi != 1.f) : (al_lo != 1.f);
     if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll
@@ -365,6 +369,12 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
         mma_bf16(o_acc[2 * dc + 1], pa[0], pa[1], pa[2], pa[3], vf[2], vf[3]);
       }
     }
+  }
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  if (kHi) {
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
   }
   cp_async_wait<0>();
   __syncthreads();
