@@ -285,18 +285,34 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       float s_odd[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
       const int mi = lane >> 3;
       const int row = wrow + (mi >> 1) * 8 + (lane & 7);
+      // all fragment loads of the slice first, then the tensor-core chain: the statements are volatile and keep their
+      // order, so loading inside the chain would expose one shared-memory latency per k-step
+      uint32_t kf[D / 16][4];
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
         const int chunk = kk * 2 + (mi & 1);
-        uint32_t kf[4];
-        ldmatrix_x4(kf, k_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
-        mma_bf16((kk & 1) ? s_odd[0] : s_acc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[0], kf[1]);
-        mma_bf16((kk & 1) ? s_odd[1] : s_acc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[2], kf[3]);
+        ldmatrix_x4(kf[kk], k_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+      }
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        mma_bf16((kk & 1) ? s_odd[0] : s_acc[0], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[kk][0], kf[kk][1]);
+        mma_bf16((kk & 1) ? s_odd[1] : s_acc[1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], kf[kk][2], kf[kk][3]);
       }
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) s_acc[j][e] += s_odd[j][e];
+      }
+    }
+    // the V fragments are fetched now, ahead of the softmax arithmetic that P V has to wait for anyway
+    uint32_t vf[D / 16][4];
+    {
+      const int mi = lane >> 3;
+      const int row = wrow + (mi & 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int dc = 0; dc < D / 16; ++dc) {
+        const int chunk = dc * 2 + (mi >> 1);
+        ldmatrix_x4_trans(vf[dc], v_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
       }
     }
     // online softmax in base 2; mask padding and skipped indices
@@ -357,17 +373,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       }
     }
     // O += P V
-    {
-      const int mi = lane >> 3;
-      const int row = wrow + (mi & 1) * 8 + (lane & 7);
 #pragma unroll
-      for (int dc = 0; dc < D / 16; ++dc) {
-        const int chunk = dc * 2 + (mi >> 1);
-        uint32_t vf[4];
-        ldmatrix_x4_trans(vf, v_st + row * kRowBytes + ((chunk ^ (row & 7)) << 4));
-        mma_bf16(o_acc[2 * dc], pa[0], pa[1], pa[2], pa[3], vf[0], vf[1]);
-        mma_bf16(o_acc[2 * dc + 1], pa[0], pa[1], pa[2], pa[3], vf[2], vf[3]);
-      }
+    for (int dc = 0; dc < D / 16; ++dc) {
+      mma_bf16(o_acc[2 * dc], pa[0], pa[1], pa[2], pa[3], vf[dc][0], vf[dc][1]);
+      mma_bf16(o_acc[2 * dc + 1], pa[0], pa[1], pa[2], pa[3], vf[dc][2], vf[dc][3]);
     }
   }
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
