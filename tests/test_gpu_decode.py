@@ -47,6 +47,9 @@ def compare(args, **kw):
     ((4096,) * 3, (100, 4096, 1), (3996, 0, 0), 8, 8, 128),   # G = 1, full budget, single token
     ((2000,), (333,), (100,), 32, 2, 128),                    # G = 16
     ((513,), (65,), (63,), 16, 2, 64),                        # G = 8, d = 64, ragged tiles
+    ((3000,), (700,), (300,), 2, 2, 64),                      # G = 1, d = 64: clusters of 8, eight outputs per owner
+    ((2500,), (350,), (150,), 4, 2, 64),                      # G = 2, d = 64, short list: 4-warp CTAs in clusters of 8
+    ((4096,) * 2, (1000,) * 2, (229,) * 2, 32, 8, 128),       # two sequences: 8-warp CTAs in clusters of 4
     ((12000,), (5000,), (3333,), 8, 2, 128),                  # few heads, long lists: clusters of 8, many slices per warp
     ((9000, 100), (4100, 10), (4500, 90), 4, 1, 128),         # one head, ragged pair of sequences
     ((25000,) * 3, (12000,) * 3, (8000,) * 3, 8, 8, 128),     # clusters of 4, long CTA ranges
