@@ -11,8 +11,9 @@
 // 16; the online softmax (base 2) stays in registers.
 // The split-KV partials (m, l, unnormalised O) never leave the chip: the warps of a CTA merge through
 // shared memory, and the CTAs of a (sequence, KV head) form a thread-block cluster (1, 2, 4 or 8 CTAs);
-// each leaves its partial in its own shared memory and, after a cluster barrier, every CTA merges a
-// slice of the G*d outputs through distributed shared memory with the log-sum-exp rule
+// every CTA owns a slice of the G*d outputs and receives the other CTAs' partials of that slice in its own
+// shared memory (remote stores that report their bytes to an mbarrier of the owner, so only the owner's merging
+// threads wait, and only for what is addressed to them), then merges them with the log-sum-exp rule
 // (m = max m_j, l = sum l_j 2^(m_j-m), o = sum o_j 2^(m_j-m) / l) and writes bf16 out and fp32 lse.
 // One launch, no workspace.
 // (Measured and dropped: a two-kernel variant with partials in HBM, 2x slower on long single-sequence

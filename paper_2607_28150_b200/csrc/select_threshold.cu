@@ -2,7 +2,7 @@
 //
 // Per (layer, sequence, KV head): the tokens whose score exceeds the row maximum minus alpha, at most cap_b
 // of them (the largest, ties to the lower index), emitted in ascending order with their count.  A threshold
-// set is an upper set of the score order, so it is the exact top-cap_b set (sg_select_topk's radix select,
+// set is an upper set of the score order, so it is the exact top-cap_b set (sg_select_topk's exact selection,
 // run first with the cap as its budget) cut at the threshold: one CTA per row finds the row maximum among the
 // cap_b candidates, keeps the candidates above max - alpha with a stable block-wide compaction in place,
 // pads the rest of the row with -1 and writes the count.  Comparisons run on the order-preserving integer

@@ -1,10 +1,12 @@
-// sg_select_topk: per-(layer, sequence, KV head) top-k by MSB-first radix select.
+// sg_select_topk: per-(layer, sequence, KV head) top-k by exact selection of the k-th largest key.
 //
-// One CTA owns one importance row.  The row's fp32 values are mapped to order-preserving uint32
-// keys and kept in shared memory (rows of up to ~55K tokens; longer rows are re-read from L2).
-// Four 8-bit histogram passes find the k-th largest key exactly; a final ordered compaction
-// (ballot + prefix counts, no atomics) emits the selected positions in ascending order, taking
-// equal-to-threshold entries from the lowest positions first.  The result is therefore a pure
+// One CTA owns one importance row.  The row's fp32 values are mapped to order-preserving uint32 keys.
+// Rows of up to 32768 tokens keep their keys in registers (second kernel below: histograms over a shrinking
+// key interval, direct ranking of the last few keys, output from bit masks; optionally fused with the gather
+// of the selected K/V rows).  Longer rows keep the keys in shared memory (up to ~55K tokens) or re-read them
+// from L2 (first kernel): four 8-bit MSB-first histogram passes find the k-th largest key exactly and a final
+// ordered compaction (ballot + prefix counts, no atomics) emits the selected positions in ascending order.
+// Both take equal-to-threshold entries from the lowest positions first.  The result is therefore a pure
 // function of the input row: identical on every run and identical to a full sort.
 #include "common.cuh"
 
