@@ -470,14 +470,26 @@ def run_ours(args):
     hp.decode_workspace(NL)
     gen_s = time.perf_counter() - t_gen
 
+    # End-to-end arm: a step's queries and local indices travel as ONE host->device copy (a staging record per step,
+    # queries first, then the index lists), as a serving loop stages the inputs of a step; the kernels read views of it.
+    q_bytes, idx_bytes = L * B * Hq * d * 2, (L * Hkv * NL * 4 if NL else 0)
+    rec = (q_bytes + idx_bytes + 255) // 256 * 256
+    h_in = torch.empty((max(nsteps_dec, 1), rec), dtype=torch.uint8).pin_memory()
+    d_in = torch.empty((max(nsteps_dec, 1), rec), dtype=torch.uint8, device=dev)
+    for s in range(nsteps_dec):
+        h_in[s, :q_bytes] = h_qdec[s].reshape(-1).view(torch.uint8)
+        if NL:
+            h_in[s, q_bytes:q_bytes + idx_bytes] = h_idx[s].reshape(-1).view(torch.uint8)
+    e_q = [d_in[s, :q_bytes].view(torch.int16).view(L, B, Hq, d) for s in range(nsteps_dec)]
+    e_idx = [d_in[s, q_bytes:q_bytes + idx_bytes].view(torch.int32).view(L, Hkv, NL) if NL else None for s in range(nsteps_dec)]
+
     def decode_all(with_copies: bool):
         for s in range(nsteps_dec):
             if with_copies:
-                d_qdec[s].copy_(h_qdec[s], non_blocking=True)
-                if NL:
-                    d_idx[s].copy_(h_idx[s], non_blocking=True)
+                d_in[s].copy_(h_in[s], non_blocking=True)
+            qs, ids = (e_q[s], e_idx[s]) if with_copies else (d_qdec[s], d_idx[s] if NL else None)
             for l in range(L):
-                hp.decode(l, d_qdec[s, l], d_k[l], d_v[l], d_idx[s, l] if NL else None, d_cu_nloc, NL, d_out[s, l])
+                hp.decode(l, qs[l], d_k[l], d_v[l], ids[l] if NL else None, d_cu_nloc, NL, d_out[s, l])
             if with_copies:
                 h_out[s].copy_(d_out[s], non_blocking=True)
 
