@@ -48,6 +48,7 @@ struct DecParams {
   int32_t* dev_status;
   int64_t ts, hs;
   int32_t B, Hq, Hkv, G, K_tot, NL_tot;
+  int32_t n_tokens;  // total tokens of the batch: with one sequence every prefix array is {0, total}, known on the host
   int32_t csize;     // CTAs per (sequence, KV head) = cluster size
   float scale_log2;
 };
@@ -153,20 +154,25 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   }
   const int b = blockIdx.x / p.csize;                          // grid.x = B * cluster size
   const int c = blockIdx.x - b * p.csize;                      // rank in the cluster
-  const int kb = p.cu_k[b + 1] - p.cu_k[b];                    // packed rows per KV head (the slot size in the buffer)
+  // A single sequence (the latency-critical case) needs no prefix loads: a dependent round trip to L2 less before the
+  // first copy can be issued.
+  const bool one = p.B == 1;
+  const int ck0 = one ? 0 : p.cu_k[b];
+  const int kb = one ? p.K_tot : p.cu_k[b + 1] - ck0;          // packed rows per KV head (the slot size in the buffer)
   const int kbe = p.packed_count ? min(kb, max(0, __ldg(p.packed_count + (int64_t)b * p.Hkv + g))) : kb;   // ... of which in the list
-  const int nl_row = p.cu_nloc[b + 1] - p.cu_nloc[b];
+  const int cl0 = one ? 0 : p.cu_nloc[b];
+  const int nl_row = one ? p.NL_tot : p.cu_nloc[b + 1] - cl0;
   const int lskip = p.local_skip ? min(nl_row, max(0, __ldg(p.local_skip + (int64_t)b * p.Hkv + g))) : 0;
   const int nl = nl_row - lskip;
-  const int c0 = p.cu[b];
-  const int nseq = p.cu[b + 1] - c0;
+  const int c0 = one ? 0 : p.cu[b];
+  const int nseq = one ? p.n_tokens : p.cu[b + 1] - c0;
   // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
   const int span = ((((kbe + nl + p.csize - 1) / p.csize) + kSlice - 1) / kSlice) * kSlice;
   const int range_beg = min(kbe + nl, c * span);
   const int range_end = min(kbe + nl, range_beg + span);
 
-  const uint16_t* pk_base = p.packed_k + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
-  const uint16_t* pv_base = p.packed_v + ((int64_t)p.cu_k[b] * p.Hkv + (int64_t)g * kb) * D;
+  const uint16_t* pk_base = p.packed_k + ((int64_t)ck0 * p.Hkv + (int64_t)g * kb) * D;
+  const uint16_t* pv_base = p.packed_v + ((int64_t)ck0 * p.Hkv + (int64_t)g * kb) * D;
   const uint16_t* lk_base = p.local_k + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
   const uint16_t* lv_base = p.local_v + (int64_t)c0 * p.ts + (int64_t)g * p.hs;
   const uint32_t wk_u32 = smem_u32(smem_raw) + warp * (kBuf * 2 * kSliceBytes);   // this warp's K ring
@@ -176,7 +182,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const int nslices = (ntok + kSlice - 1) / kSlice;
   // warp w streams slices w, w + kDecWarps, ... of the range, so the CTA walks memory front to back
   const int nmine = nslices > warp ? (nslices - warp + kDecWarps - 1) / kDecWarps : 0;
-  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + p.cu_nloc[b] + lskip - kbe;   // indexed by list position
+  const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + cl0 + lskip - kbe;   // indexed by list position
   // Lane r (and r + 16) holds the local index of row r of the warp's j-th slice, read one slice ahead.
   auto fetch_idx = [&](int j) -> int {
     const int li = (warp + j * kDecWarps) * kSlice + (lane & 15);
@@ -596,6 +602,7 @@ sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed
   p.G = G;
   p.K_tot = total_sel;
   p.NL_tot = total_loc;
+  p.n_tokens = shape->total_tokens;
   int warps = 4;
   decode_plan(shape, total_sel, total_loc, &p.csize, &warps);
   p.scale_log2 = (softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D)) * kLog2e;
