@@ -191,6 +191,22 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   };
   auto load_slice = [&](int j, int buf, int idx_reg) {
     const int li0 = (warp + j * kDecWarps) * kSlice;
+    if (li0 + kSlice <= ntok && pos_beg + li0 + kSlice <= kbe) {
+      // the whole slice lies in the packed buffer: 16 consecutive rows are one contiguous run of 16-byte pieces
+      if (lane == 0) s_mask[warp * kBuf + buf] = 0xffffu;
+      const uint16_t* srck = pk_base + (int64_t)(pos_beg + li0) * D + lane * 8;
+      const uint16_t* srcv = pv_base + (int64_t)(pos_beg + li0) * D + lane * 8;
+#pragma unroll
+      for (int i = 0; i < kCopiesPerLane; ++i) {
+        const int qid = lane + i * 32;
+        const int row = qid / kChunksPerRow;
+        const int col = qid % kChunksPerRow;
+        const uint32_t off = buf * kSliceBytes + row * kRowBytes + ((col ^ (row & 7)) << 4);
+        cp_async16(wk_u32 + off, srck + i * 256, 16);
+        cp_async16(wv_u32 + off, srcv + i * 256, 16);
+      }
+      return;
+    }
     {
       const int li = li0 + (lane & 15), pos = pos_beg + li;
       const bool in_list = li < ntok;
@@ -238,9 +254,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
 #pragma unroll
     for (int s = 0; s < kBuf - 1; ++s) idx_pro[s] = fetch_idx(s);
     idx_next = fetch_idx(kBuf - 1);
-#pragma unroll
-    for (int s = 0; s < kBuf - 1; ++s) {
-      if (s < nmine) load_slice(s, s, idx_pro[s]);
+    static_assert(kBuf == 3, "the prologue below passes two index registers by selection");
+#pragma unroll 1
+    for (int s = 0; s < kBuf - 1; ++s) {                      // not unrolled: this code runs once per call, from a cold instruction cache
+      if (s < nmine) load_slice(s, s, s ? idx_pro[1] : idx_pro[0]);
       cp_async_commit();
     }
   }
