@@ -2,9 +2,9 @@
 //
 // Memory-bound: every attended token costs 2*d*2 bytes of K+V per KV head and only 4*G*d flops.
 // The token list of a (sequence, KV head) -- packed rows first, then local rows addressed through
-// local_idx -- is cut into slices of 16 tokens.  The CTAs that share a (sequence, KV head) split the list
-// evenly; inside a CTA warp w takes slices w, w + warps, ... and streams them through a ring of three
-// K/V slices of its own in shared memory (16-byte cp.async copies, XOR-swizzled rows so ldmatrix is
+// local_idx -- is cut into slices of 16 tokens.  The slices are dealt out round robin over all warps of all
+// CTAs that share a (sequence, KV head), so every CTA gets the same mix of packed and gathered slices; a warp
+// streams its slices through a ring of three K/V slices of its own in shared memory (16-byte cp.async copies, XOR-swizzled rows so ldmatrix is
 // conflict-free; gathered rows are whole 2*d-byte lines, so sector efficiency stays 100 %).  The ring is
 // private to the warp, so the loop has no block-wide barrier: a warp waits only for its own copies.
 // S = Q K^T and O += P V run on bf16 tensor-core MMAs with the G query rows of the KV head padded to
@@ -166,10 +166,6 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const int nl = nl_row - lskip;
   const int c0 = one ? 0 : p.cu[b];
   const int nseq = one ? p.n_tokens : p.cu[b + 1] - c0;
-  // token range of this CTA within the list [packed rows ++ local rows] of (b, g)
-  const int span = ((((kbe + nl + p.csize - 1) / p.csize) + kSlice - 1) / kSlice) * kSlice;
-  const int range_beg = min(kbe + nl, c * span);
-  const int range_end = min(kbe + nl, range_beg + span);
 
   const uint16_t* pk_base = p.packed_k + ((int64_t)ck0 * p.Hkv + (int64_t)g * kb) * D;
   const uint16_t* pv_base = p.packed_v + ((int64_t)ck0 * p.Hkv + (int64_t)g * kb) * D;
@@ -178,19 +174,23 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   const uint32_t wk_u32 = smem_u32(smem_raw) + warp * (kBuf * 2 * kSliceBytes);   // this warp's K ring
   const uint32_t wv_u32 = wk_u32 + kBuf * kSliceBytes;                            // and its V ring
 
-  const int pos_beg = range_beg, ntok = range_end - range_beg;
+  // The slices of the list [packed rows ++ local rows] of (b, g) are dealt out round robin over all warps of all CTAs of
+  // the cluster (slice s goes to rank s % csize, warp (s / csize) % warps): every CTA gets the same mix of contiguous
+  // packed slices and slower gathered ones, whatever the split of the list.
+  constexpr int pos_beg = 0;
+  const int ntok = kbe + nl;
   const int nslices = (ntok + kSlice - 1) / kSlice;
-  // warp w streams slices w, w + kDecWarps, ... of the range, so the CTA walks memory front to back
-  const int nmine = nslices > warp ? (nslices - warp + kDecWarps - 1) / kDecWarps : 0;
+  const int first_slice = warp * p.csize + c, slice_stride = kDecWarps * p.csize;
+  const int nmine = nslices > first_slice ? (nslices - first_slice + slice_stride - 1) / slice_stride : 0;
   const int32_t* idx_base = p.local_idx + (int64_t)g * p.NL_tot + cl0 + lskip - kbe;   // indexed by list position
   // Lane r (and r + 16) holds the local index of row r of the warp's j-th slice, read one slice ahead.
   auto fetch_idx = [&](int j) -> int {
-    const int li = (warp + j * kDecWarps) * kSlice + (lane & 15);
+    const int li = (first_slice + j * slice_stride) * kSlice + (lane & 15);
     const int pos = pos_beg + li;
     return (j < nmine && li < ntok && pos >= kbe) ? __ldg(idx_base + pos) : 0;
   };
   auto load_slice = [&](int j, int buf, int idx_reg) {
-    const int li0 = (warp + j * kDecWarps) * kSlice;
+    const int li0 = (first_slice + j * slice_stride) * kSlice;
     if (li0 + kSlice <= ntok && pos_beg + li0 + kSlice <= kbe) {
       // the whole slice lies in the packed buffer: 16 consecutive rows are one contiguous run of 16-byte pieces
       if (lane == 0) s_mask[warp * kBuf + buf] = 0xffffu;
