@@ -531,6 +531,8 @@ void decode_plan(const sg_shape* shape, int32_t total_sel, int32_t total_loc, in
     int work = 1;
     while (work < 8 && (int64_t)work * W * kSlice < avg_tokens) work *= 2;
     cs = fit < work ? fit : work;
+    // many short lists: one 8-warp CTA per list has a slice or two per warp already, and no cluster to merge
+    if (pairs >= 64 && avg_tokens <= 14 * kSlice) { W = 8; cs = 1; }
   } else {
     auto fill = [&](int64_t slots) { return (double)pairs / (double)(((pairs + slots - 1) / slots) * slots); };
     W = (avg_tokens >= 1024 && fill(kNumSMs) > fill(2 * kNumSMs) + 0.05) ? 8 : 4;
