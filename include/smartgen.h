@@ -151,6 +151,9 @@ sg_status sg_select_pack_kv(const sg_shape* shape, const float* importance, cons
  * packed_k/v  bf16 [K_tot*H_kv][d], layout of sg_pack_kv for one layer; cu_k as in sg_pack_kv.
  * local_k/v   bf16, element (token, g, c) at token*token_stride + g*head_stride + c.
  * local_idx   int32 [H_kv][NL_tot]; cu_nloc device int32 [B+1]; total_loc = cu_nloc[B].
+ *             The host totals are binding: with one sequence (B = 1) the kernel takes k_0 = total_sel,
+ *             n_loc_0 = total_loc and N_0 = shape->total_tokens from the arguments and does not read the
+ *             prefix arrays at all (they must still be valid pointers that hold {0, total}).
  * softmax_scale  0 means 1/sqrt(d).
  * out         bf16 [B][H_q][d]; lse fp32 [B][H_q] (may be NULL) = max + ln(sum) of the scaled
  *             scores.  A head with an empty list gets out = 0 and lse = -inf.
