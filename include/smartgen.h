@@ -93,14 +93,18 @@ sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache
  * (Section 2.3, BH x k KV index).  For every (l, b, g) the k_b = cu_k[b+1] - cu_k[b] positions
  * of sequence b with the largest importance are kept.  Order of values: the total order of the
  * fp32 bit patterns (+0 above -0, +inf above every finite value -- so entries given infinite
- * importance as in Eq. 1 are always kept); equal values go to the lower position.  Each row is
- * emitted in ascending position order (entry order does not change attention, Section 4.2).
+ * importance as in Eq. 1 are always kept); equal values go to the lower position.  NaNs take the
+ * place their bit patterns have in that order: a NaN with a clear sign bit ranks above +inf, one with
+ * a set sign bit below -inf, two NaNs by payload (sg_score never produces a NaN from finite inputs).
+ * Each row is emitted in ascending position order (entry order does not change attention, Section 4.2).
  *
  * importance  fp32 [L][H_kv][T].
  * cu_k        device int32 [B+1], prefix sums of k_b; total_sel = cu_k[B] (host copy of the total).
  * sel_idx     int32 [L][H_kv][K_tot]; the row segment of (l, g, b) starts at cu_k[b]; positions
  *             are sequence-local (0 .. N_b-1).  k_b > N_b sets the SG_ERR_INVALID device bit and
- *             the row is filled with 0 .. N_b-1 followed by -1.
+ *             the row is filled with 0 .. N_b-1 followed by -1.  A sequence longer than
+ *             shape->max_seqlen (which sizes the kernel's key storage) sets the same bit and its
+ *             rows are filled with -1; nothing outside the provided buffers is touched.
  */
 sg_status sg_select_topk(const sg_shape* shape, const float* importance, const int32_t* cu_k,
                          int32_t total_sel, int32_t* sel_idx, void* workspace, size_t workspace_bytes,

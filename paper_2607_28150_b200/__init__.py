@@ -13,7 +13,7 @@ __all__ = ["binding", "workloads", "build"]
 
 
 def __getattr__(name):
-    if name in ("binding", "workloads", "build", "smoke", "pipeline", "replicas"):
+    if name in ("binding", "workloads", "build", "pipeline", "replicas"):
         return importlib.import_module(__name__ + "." + name)
     if name.startswith("sg_") or name.startswith("SG_") or name in ("Shape", "SmartGenError"):
         return getattr(importlib.import_module(__name__ + ".binding"), name)

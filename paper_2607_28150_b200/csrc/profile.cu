@@ -1,7 +1,7 @@
 // Profile-based proactive selection on the device: selection counts S(e), block importance (Eq. 1), the
 // transfer budget (Eq. 2, host arithmetic) and the KV mask left by the proactive transfer.  The global
 // top-K_r over the L*M block importances is sg_select_topk on the flattened matrix.  Integer work plus one
-// double division per block; every result is bit-exact against the oracle.
+// double division per block; every result is bit-exact against a scalar fp64 CPU restatement of the equations.
 #include <math.h>
 
 #include "common.cuh"

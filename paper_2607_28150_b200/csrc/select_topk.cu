@@ -28,6 +28,7 @@ struct SelParams {
   int32_t* dev_status;
   int64_t T;
   int32_t K_tot, B, Hkv;
+  int32_t capacity;        // longest row the launched kernel variant can hold (from shape->max_seqlen); 0 = any length
   // fused packing (select_topk_reg_kernel with PD > 0): the CTA that selected a row also gathers its K/V rows
   const uint16_t* k_cache;
   const uint16_t* v_cache;
@@ -66,6 +67,13 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelPa
   const int kb = p.cu_k[b + 1] - ck;
   if (kb <= 0) return;
   int32_t* out = p.sel_idx + ((int64_t)l * p.Hkv + g) * p.K_tot + ck;
+  if (p.capacity > 0 && N > p.capacity) {
+    // The row is longer than the shape's max_seqlen promised (the key array was sized from it): flag it and
+    // emit an empty row instead of touching memory the launch did not provide.
+    if (tid == 0) raise(p.dev_status, SG_ERR_INVALID);
+    for (int j = tid; j < kb; j += kSelThreads) out[j] = -1;
+    return;
+  }
   if (kb >= N) {                                      // whole prompt (or an over-sized budget)
     if (kb > N && tid == 0) raise(p.dev_status, SG_ERR_INVALID);
     for (int j = tid; j < kb; j += kSelThreads) out[j] = j < N ? j : -1;
@@ -263,6 +271,17 @@ __global__ void __launch_bounds__(T) select_topk_reg_kernel(const SelParams p) {
       }
     }
   };
+  if (N > p.capacity) {
+    // Longer than the E*T positions this variant holds (it was chosen from shape->max_seqlen, which the row
+    // exceeds): flag it, emit an empty row (and zero rows in the fused gather) and leave.
+    if (tid == 0) {
+      raise(p.dev_status, SG_ERR_INVALID);
+      if (PD > 0) raise(p.dev_status, SG_ERR_INDEX);
+    }
+    for (int j = tid; j < kb; j += T) out[j] = -1;
+    pack_rows([&](int) { return -1; });
+    return;
+  }
   if (kb >= N) {                                      // whole prompt (or an over-sized budget)
     if (kb > N && tid == 0) {
       raise(p.dev_status, SG_ERR_INVALID);
@@ -447,6 +466,7 @@ sg_status select_launch(const sg_shape* shape, SelParams& p, bool fuse, void* st
   const int pd = fuse ? shape->head_dim : 0;
 #define SG_LAUNCH_SELECT_REG_PD(E, T, PD)                                                       \
   do {                                                                                          \
+    p.capacity = (E) * (T);                                                                     \
     SG_ENSURE_SMEM((select_topk_reg_kernel<E, T, PD>), (select_reg_smem_bytes<E, T>()));         \
     select_topk_reg_kernel<E, T, PD><<<(unsigned)rows, T, select_reg_smem_bytes<E, T>(), s>>>(p); \
   } while (0)
@@ -471,9 +491,11 @@ sg_status select_launch(const sg_shape* shape, SelParams& p, bool fuse, void* st
     return SG_ERR_UNSUPPORTED;
   } else if (shape->max_seqlen <= kSelKeyCap) {
     const int smem = kSelFixedSmem + shape->max_seqlen * 4;
+    p.capacity = shape->max_seqlen;
     SG_ENSURE_SMEM(select_topk_kernel<true>, smem);
     select_topk_kernel<true><<<(unsigned)rows, kSelThreads, smem, s>>>(p);
   } else {
+    p.capacity = 0;                                    // keys are re-read from global memory: any length
     select_topk_kernel<false><<<(unsigned)rows, kSelThreads, kSelFixedSmem, s>>>(p);
   }
 #undef SG_LAUNCH_SELECT_REG

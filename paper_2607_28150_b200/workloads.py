@@ -2,7 +2,7 @@
 
 This module only *shapes inputs*.  It holds none of the method's arithmetic (no
 scoring, no selection, no attention) and imports neither the CUDA binding nor
-the CPU oracle, so the same arrays can be fed to both sides of a parity test.
+any CPU checker, so the same arrays can be fed to both sides of a parity test.
 
 Everything is numpy with a counter-based generator (``Philox``), keyed by
 ``(config id, layer, tensor id)``, so any layer of any configuration can be

@@ -82,3 +82,58 @@ def test_select_narrow_clustered_and_wide_key_ranges():
     wide[:, :, 5::101] = -np.float32(np.inf)
     check(wide, (n,), (1000,))
     check(wide, (4096, 4096), (4000, 2))
+
+
+def test_select_nan_ordered_by_bit_pattern():
+    """NaNs rank where their bit patterns put them (clear sign bit: above +inf; set sign bit: below -inf), on every
+    kernel variant: registers (8 / 16 / 32 keys per thread), keys in shared memory, keys re-read from global memory."""
+    rng = np.random.default_rng(11)
+    for n, k in ((3000, 100), (8192, 820), (30000, 2500), (40000, 3000), (60000, 500)):
+        x = rng.standard_normal((1, 2, n)).astype(np.float32)
+        xb = x.view(np.uint32)
+        xb[0, :, ::13] = 0x7FC00000 | rng.integers(0, 1 << 22, size=xb[0, :, ::13].shape).astype(np.uint32)
+        xb[0, :, 5::17] = 0xFFC00000 | rng.integers(0, 1 << 22, size=xb[0, :, 5::17].shape).astype(np.uint32)
+        xb[0, :, 7::19] = 0x7F800001                      # signalling NaN with the smallest payload
+        check(x, (n,), (k,))
+        check(x, (n,), (n - 3,))                          # the negative NaNs are the ones left out
+
+
+def test_select_row_longer_than_max_seqlen_is_flagged_not_read():
+    """shape->max_seqlen sizes the kernels' key storage.  A sequence longer than it must set SG_ERR_INVALID and get
+    an empty row (-1), with no access outside the buffers, in the selection, the fused selection + gather, and the
+    shared-memory variant; the other sequences of the batch are selected as usual."""
+    import torch
+    import gpu_ops
+    import paper_2607_28150_b200.binding as sg
+    rng = np.random.default_rng(12)
+    for lens, ks, lie, L, Hkv in (((3000, 9000), (30, 90), 4096, 1, 2), ((1000, 9000), (10, 90), 4096, 10, 8),
+                                  ((1000, 50000), (10, 100), 34000, 1, 1)):
+        cu, ck = cu_of(lens), cu_of(ks)
+        T, Kt, d = int(cu[-1]), int(ck[-1]), 64
+        x = rng.random((L, Hkv, T), dtype=np.float32)
+        shp = sg.make_shape(L, Hkv, Hkv, d, 1, gpu_ops.dev(cu), T, lie)
+        want = oracle.select_topk(x, cu, ck)
+        want[:, :, ck[1]:ck[2]] = -1
+        sel = gpu_ops.Guarded((L, Hkv, Kt), torch.int32, -99)
+        st = gpu_ops.status_word()
+        sg.sg_select_topk(shp, gpu_ops.dev(x), gpu_ops.dev(ck), Kt, sel.view, None, st)
+        assert np.array_equal(sel.numpy(), want)
+        assert gpu_ops.read_status(st) == 1 << sg.SG_ERR_INVALID
+        if lie > 32768:
+            continue
+        k = rng.integers(0, 1 << 16, size=(L, T, Hkv, d), dtype=np.uint16)
+        v = rng.integers(0, 1 << 16, size=(L, T, Hkv, d), dtype=np.uint16)
+        sel = gpu_ops.Guarded((L, Hkv, Kt), torch.int32, -99)
+        pk = gpu_ops.Guarded((L, Kt * Hkv, d), torch.int16, 0x5555)
+        pv = gpu_ops.Guarded((L, Kt * Hkv, d), torch.int16, 0x5555)
+        st = gpu_ops.status_word()
+        sg.sg_select_pack_kv(shp, gpu_ops.dev(x), gpu_ops.dev(ck), Kt, gpu_ops.dev(k), gpu_ops.dev(v), sel.view, pk.view,
+                             pv.view, st)
+        assert np.array_equal(sel.numpy(), want)
+        assert gpu_ops.read_status(st) == (1 << sg.SG_ERR_INVALID) | (1 << sg.SG_ERR_INDEX)
+        safe = np.where(want < 0, 0, want)
+        pk_o, pv_o = oracle.pack_kv(k, v, cu, safe, ck)
+        rows = slice(ck[1] * Hkv, ck[2] * Hkv)
+        pk_o[:, rows] = 0
+        pv_o[:, rows] = 0
+        assert np.array_equal(pk.numpy(), pk_o) and np.array_equal(pv.numpy(), pv_o)

@@ -62,13 +62,31 @@ def test_split_without_reordering_keeps_row_order_and_drops_padding():
             assert rem[g, ck[b]: ck[b] + nr[b, g]].tolist() == row[m == 2].tolist()
 
 
-def test_mask_footprint_matches_printed_example():
+def test_kv_mask_of_the_printed_example_has_the_printed_footprint():
+    """Section 4.2 prints the cost of the KV mask for 64K tokens on a 40-layer model: one int8 per token and layer,
+    2.5 MB in all.  The masks the oracle builds (proactive transfer of the global top blocks, one mask per layer)
+    must have exactly that footprint, hold only the classes 1 / 2, and be the structure Algorithm 1 indexes."""
     path = os.path.join(os.path.dirname(__file__), "golden", "kv_mask_footprint.txt")
     rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
     tokens, layers, per_layer, total_mb = int(rows[0][0]), int(rows[0][1]), int(rows[0][2]), float(rows[0][3])
-    mask = np.zeros(tokens, dtype=np.int8)            # the mask the oracle indexes: one int8 per token
-    assert mask.nbytes == per_layer == 64 * 1024
-    assert layers * mask.nbytes / 2**20 == total_mb
+    cu = np.array([0, tokens], dtype=np.int32)
+    M = 64
+    selected = np.arange(0, layers * M, 3, dtype=np.int32)          # every third block, ascending flat ids
+    masks = [oracle.proactive_mask(cu, M, l, selected) for l in range(layers)]
+    assert all(m.dtype == np.int8 and m.shape == (tokens,) for m in masks)
+    assert masks[0].nbytes == per_layer
+    assert sum(m.nbytes for m in masks) / 2**20 == total_mb
+    for l in (0, 1, layers - 1):
+        blocks = (np.arange(tokens, dtype=np.int64) * M) // tokens
+        want = np.where(np.isin(l * M + blocks, selected), 1, 2).astype(np.int8)
+        assert np.array_equal(masks[l], want)
+    # the same mask drives Algorithm 1 at that size: a row of indices splits into the two classes it marks
+    idx = np.arange(0, tokens, 97, dtype=np.int32)[None, :]
+    ck = np.array([0, idx.shape[1]], dtype=np.int32)
+    _, loc, rem, nl, nr = oracle.split_index(idx, masks[2], cu, ck, reorder=False)
+    assert nl[0, 0] + nr[0, 0] == idx.shape[1]
+    assert loc[0, : nl[0, 0]].tolist() == idx[0][masks[2][idx[0]] == 1].tolist()
+    assert rem[0, : nr[0, 0]].tolist() == idx[0][masks[2][idx[0]] == 2].tolist()
 
 
 def test_two_lane_fetching_equals_attention_over_the_kv_index():

@@ -99,3 +99,34 @@ def test_topk_hypothesis_few_distinct_values(vals, data):
 def test_topk_rejects_budget_above_length():
     with pytest.raises(RuntimeError):
         run(np.zeros((1, 1, 4), dtype=np.float32), (4,), (5,))
+
+
+def _nan(sign, payload):
+    """A float32 NaN with the given sign bit and mantissa payload (non-zero)."""
+    return np.array([(sign << 31) | 0x7F800000 | payload], dtype=np.uint32).view(np.float32)[0]
+
+
+def test_topk_nan_takes_the_place_of_its_bit_pattern():
+    """The order of values is the total order of the fp32 bit patterns: a NaN with a clear sign bit ranks above
+    +inf (larger payload first), one with a set sign bit below -inf.  Restated here with plain integers: the rank of a
+    value is its sign-magnitude pattern read as a signed quantity."""
+    vals = np.array([1.0, _nan(0, 1), np.inf, _nan(0, 0x400000), -np.inf, _nan(1, 1), 0.0, _nan(1, 0x400000), -2.0, 1.0],
+                    dtype=np.float32)
+    bits = vals.view(np.uint32).astype(np.int64)
+    rank = np.where(bits >> 31 == 1, -(bits & 0x7FFFFFFF) - 1, bits & 0x7FFFFFFF)      # -0 just below +0
+    order = sorted(range(len(vals)), key=lambda t: (-int(rank[t]), t))
+    assert order[:3] == [3, 1, 2] and order[-2:] == [5, 7]                         # quiet NaN, NaN(1), +inf ... -NaNs last
+    for k in range(len(vals) + 1):
+        sel, _, _ = run(vals[None, None], (len(vals),), (k,))
+        assert sel[0, 0].tolist() == sorted(order[:k])
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((1, 2, 300)).astype(np.float32)
+    xb = x.view(np.uint32)
+    xb[0, :, ::7] = 0x7FC00000 | rng.integers(0, 1 << 22, size=xb[0, :, ::7].shape).astype(np.uint32)
+    xb[0, :, 3::11] = 0xFFC00000 | rng.integers(0, 1 << 22, size=xb[0, :, 3::11].shape).astype(np.uint32)
+    sel, cu, ck = run(x, (300,), (60,))
+    for g in range(2):
+        b_ = x[0, g].view(np.uint32).astype(np.int64)
+        r_ = np.where(b_ >> 31 == 1, -(b_ & 0x7FFFFFFF) - 1, b_ & 0x7FFFFFFF)
+        want = sorted(sorted(range(300), key=lambda t: (-int(r_[t]), t))[:60])
+        assert sel[0, g].tolist() == want
