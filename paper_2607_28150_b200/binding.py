@@ -22,7 +22,8 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 # every symbol include/smartgen.h declares
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
             "sg_score_static", "sg_select_pack_kv", "sg_select_threshold", "sg_pack_kv_counted", "sg_sparse_decode_attn_counted", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
-            "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error")
+            "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error",
+            "sg_testing_score_fault", "sg_testing_score_clock", "sg_testing_score_grid")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -89,6 +90,29 @@ _lib.sg_split_index.argtypes = [_sp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp, _
 _lib.sg_sparse_decode_attn.restype = ctypes.c_int
 _lib.sg_sparse_decode_attn.argtypes = [_sp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp,
                                        _sz, _vp, _vp]
+
+
+_lib.sg_testing_score_fault.restype = None
+_lib.sg_testing_score_fault.argtypes = [_i32, _i32]
+_lib.sg_testing_score_clock.restype = None
+_lib.sg_testing_score_clock.argtypes = [_vp]
+_lib.sg_testing_score_grid.restype = _i32
+_lib.sg_testing_score_grid.argtypes = [_sp]
+
+
+def sg_testing_score_fault(withhold_unit: int = -1, wait_limit_ms: int = 0) -> None:
+    """Test hook: withhold the done-count of one scoring unit and/or shorten every bounded wait (0 / -1 = off)."""
+    _lib.sg_testing_score_fault(withhold_unit, wait_limit_ms)
+
+
+def sg_testing_score_clock(buffer: Optional[torch.Tensor]) -> None:
+    """Measurement hook: the next scoring kernels record their start/end clock64 and globaltimer per CTA into
+    `buffer` (int64, at least 32 words per CTA); None switches it off."""
+    _lib.sg_testing_score_clock(None if buffer is None else buffer.data_ptr())
+
+
+def sg_testing_score_grid(shape: "Shape") -> int:
+    return int(_lib.sg_testing_score_grid(ctypes.byref(shape)))
 
 
 def make_shape(num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,

@@ -26,6 +26,12 @@ NVCC_FLAGS = [
 ]
 
 
+# Extra nvcc flags for a debug or profiling build of the whole library, e.g. SG_NVCC_FLAGS="-DSG_SCORE_PROFILE";
+# such a build always recompiles, and so does the next ordinary one.
+EXTRA_FLAGS = os.environ.get("SG_NVCC_FLAGS", "").split()
+_STAMP = os.path.join(OBJDIR, "flags.txt")
+
+
 def _nvcc() -> str:
     cand = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(cand):
@@ -40,7 +46,7 @@ def _newest_dep() -> float:
 
 
 def _compile(src: str, obj: str, verbose: bool) -> None:
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+    cmd = [_nvcc()] + NVCC_FLAGS + EXTRA_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (src, res.stdout, res.stderr))
@@ -53,6 +59,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not srcs:
         raise RuntimeError("no CUDA sources under %s" % CSRC)
     os.makedirs(OBJDIR, exist_ok=True)
+    last = open(_STAMP).read() if os.path.exists(_STAMP) else ""
+    if last != " ".join(EXTRA_FLAGS):
+        force = True                                     # objects on disk were built with other flags
     dep_time = _newest_dep()
     jobs, objs = [], []
     for s in srcs:
@@ -71,6 +80,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if res.returncode != 0:
             raise RuntimeError("link failed:\n%s\n%s" % (res.stdout, res.stderr))
         os.replace(tmp, LIB)
+    with open(_STAMP, "w") as f:
+        f.write(" ".join(EXTRA_FLAGS))
     return LIB
 
 

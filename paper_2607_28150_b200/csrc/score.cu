@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include <vector>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "launch.h"
@@ -37,7 +38,12 @@ namespace {
 
 constexpr int kEpiGroups = 4;             // epilogue warpgroups (four warps each, one per TMEM lane quarter)
 constexpr int kEpiThreads = 128 * kEpiGroups;
-constexpr int kScoreThreads = 64 + kEpiThreads;   // warp 0: TMA, warp 1: MMA + TMEM owner, then the epilogue warps
+// Warp roles: warps 0-15 are the epilogue (four hardware-aligned warpgroups), warp 16 feeds TMA, warp 17 issues the MMAs and owns the TMEM allocation, warps 18 and 19 (the helpers)
+// merge row statistics off the epilogue's path.
+constexpr int kTmaWarp = kEpiThreads / 32;
+constexpr int kMmaWarp = kTmaWarp + 1;
+constexpr int kHelperWarp = kTmaWarp + 2;
+constexpr int kScoreThreads = kEpiThreads + 128;
 constexpr int kTileKeys = 128;
 constexpr int kRing = 4 / kEpiGroups;        // accumulator stages per epilogue warpgroup
 constexpr int kAccStages = 4;             // 4 x 128 fp32 columns = the whole 512-column TMEM
@@ -47,12 +53,31 @@ constexpr int kMaxKStages = 4;
 constexpr int kSmemLimit = 232448;        // 227 KB opt-in dynamic shared memory per CTA
 constexpr float kLog2e = 1.4426950408889634f;
 
+// Profiling build (-DSG_SCORE_PROFILE): selected threads add up the clocks they spend in each kind of wait and
+// write the sums behind the CTA's four clock words of the testing clock buffer (32 words per CTA).
+#ifdef SG_SCORE_PROFILE
+#define SG_PROF_DECL(...) long long __VA_ARGS__
+#define SG_PROF_BEGIN(t) const long long t = clock64()
+#define SG_PROF_ADD(acc, t) acc += clock64() - (t)
+#define SG_PROF_INC(acc) acc += 1
+#define SG_PROF_EVENT(kind, n) do { if (p.clock_out && blockIdx.x == 0 && (n) < 4096u) p.clock_out[32 * 1024 + (kind) * 4096 + (n)] = (unsigned long long)clock64(); } while (0)
+#define SG_PROF_STORE(slot, v) do { if (p.clock_out) p.clock_out[32 * (size_t)blockIdx.x + (slot)] = (unsigned long long)(v); } while (0)
+constexpr int kClockWords = 32;
+#else
+#define SG_PROF_DECL(...)
+#define SG_PROF_BEGIN(t)
+#define SG_PROF_ADD(acc, t)
+#define SG_PROF_INC(acc)
+#define SG_PROF_EVENT(kind, n)
+#define SG_PROF_STORE(slot, v)
+constexpr int kClockWords = 4;
+#endif
+
 struct ScoreParams {
   const int32_t* cu;
   float* importance;
   int* p1_done;            // [U] pass-1 items finished per unit (zeroed by the host call)
-  float* part_m;           // [U][max_items][Ralloc] per-item row statistics (log2 domain max, sum)
-  float* part_l;
+  float2* part;            // [U][max_items][Ralloc] per-item row statistics (log2-domain max, sum of exp2)
   int32_t* dev_status;
   int64_t T;
   int32_t B, Hkv, G, W, R, Rpad, Ralloc;
@@ -60,6 +85,11 @@ struct ScoreParams {
   int32_t lag;             // pass 2 of unit u is scheduled `lag` units after its pass 1
   int32_t compact;         // schedule layout: 0 = every slot 2*C positions, 1 = positions without an item removed
   int32_t tiles_per_chunk, max_items, k_stages, q_bufs;
+  int32_t wgslots;         // statistics slots per item: 4 (one per epilogue warpgroup) or 1 (every row block has one owner)
+  int32_t debug_mode;      // profiling builds only: 1 = epilogue releases accumulators without reading them
+  int32_t withhold_unit;   // testing only: pass-1 items of this unit are never counted as done (-1 = none)
+  uint32_t wait_ns;        // limit of every bounded wait, nanoseconds
+  unsigned long long* clock_out;   // testing only: per CTA {clock64 start, end, globaltimer start, end}, or null
   float scale_log2;
 };
 
@@ -78,23 +108,36 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: gives up after about one second, or as soon as another thread has set *abort_flag.
-// try_wait is given a suspend-time hint, so a waiting thread sleeps in hardware (and is woken when the phase
-// completes) instead of spinning through the issue slots the working warps need.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// One try_wait: true when the phase has completed.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after `limit_ns` (about one second in normal use), or once another thread has set
+// *abort_flag.  try_wait comes back after a short, hardware-chosen time whether or not the phase has completed, so a
+// thread that simply retries spins through a dozen instructions per attempt -- issue slots and, worse, entries of the
+// queue that the SFU instructions of the working warps go through (measured: one retry per 11 clocks and SM, 60 % of
+// all executed instructions, SFU pipe at 51 %).  A waiter therefore sleeps `sleep_ns` between attempts (chosen per
+// role: short on the MMA thread's critical path, long for the producer that runs ahead) and looks at the clock and the
+// abort flag only every 64th attempt.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit_ns,
+                                          uint32_t sleep_ns) {
+  if (mbar_test(bar, parity)) return true;
   uint64_t t0 = 0;
-  for (;;) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(200000u) : "memory");
-    if (ok) return true;
-    if (*abort_flag) return false;
-    const uint64_t now = global_timer_ns();
-    if (t0 == 0) t0 = now;
-    else if (now - t0 > 1000000000ull) { *abort_flag = 1; return false; }
+  for (uint32_t it = 0;; ++it) {
+    if (sleep_ns) __nanosleep(sleep_ns);
+    if (mbar_test(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > (uint64_t)limit_ns) { *abort_flag = 1; return false; }
+    }
   }
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -136,24 +179,81 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32
         ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
   }
 }
+// All MMAs of one accumulator block in a single statement: NK k-steps of 16 elements, four per 128-byte
+// sub-tile (descriptor low word += 2 per step inside a sub-tile, += a_sub / b_sub to the next sub-tile).  The first
+// MMA overwrites the accumulator, the others add to it.  One statement keeps the issuing thread's instruction
+// stream to the bare minimum between two blocks: the tensor pipe drains its short queue within ~200 clocks of the
+// last issue, so every clock spent between blocks is an idle clock of the pipe.
+template <int NK>
+__device__ __forceinline__ void umma_block(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t a_sub, uint32_t b_sub,
+                                           uint32_t desc_hi, uint32_t idesc) {
+  static_assert(NK == 4 || NK == 8, "one or two 64-element sub-tiles along d");
+  if (NK == 8) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .b32 a, b;\n\t.reg .pred pf, pt;\n\t"
+        "setp.ne.u32 pf, %0, %0;\n\tsetp.eq.u32 pt, %0, %0;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pf;\n\t"
+        "add.u32 a, %1, 2;\n\tadd.u32 b, %2, 2;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, %1, 4;\n\tadd.u32 b, %2, 4;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, %1, 6;\n\tadd.u32 b, %2, 6;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, %1, %3;\n\tadd.u32 b, %2, %4;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, a, 2;\n\tadd.u32 b, b, 2;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, a, 2;\n\tadd.u32 b, b, 2;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t"
+        "add.u32 a, a, 2;\n\tadd.u32 b, b, 2;\n\tmov.b64 da, {a, %5};\n\tmov.b64 db, {b, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %6, pt;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(a_sub), "r"(b_sub), "r"(desc_hi), "r"(idesc) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .b32 a, b;\n\t.reg .pred pf, pt;\n\t"
+        "setp.ne.u32 pf, %0, %0;\n\tsetp.eq.u32 pt, %0, %0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
+        "add.u32 a, %1, 2;\n\tadd.u32 b, %2, 2;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+        "add.u32 a, %1, 4;\n\tadd.u32 b, %2, 4;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+        "add.u32 a, %1, 6;\n\tadd.u32 b, %2, 6;\n\tmov.b64 da, {a, %3};\n\tmov.b64 db, {b, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
+  }
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// TMEM load of 32 consecutive fp32 columns of this thread's lane, complete on return (load and wait are one
-// asm statement, so the compiler sees plain outputs).
-__device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
+// TMEM load of 32 consecutive fp32 columns of this thread's lane, issued without waiting: the registers hold
+// the data only after tmem_ld_wait().  A warp issues the load of its next 32 columns before it works on the
+// current ones, so the load's latency is covered by arithmetic.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t (&r)[32], uint32_t taddr) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+// Waits for the thread's outstanding TMEM loads.  The empty statements that follow tie the 32 registers of the
+// load that has just completed to this point of the program: volatile statements keep their order, and every
+// later use of the registers depends on them, so the compiler cannot schedule arithmetic on the data ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; i += 8)
+    asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
+                      "+r"(r[i + 6]), "+r"(r[i + 7]) :: "memory");
+}
+// Barrier among the 128 threads of one epilogue warpgroup (named barriers 2..5); no CTA-wide barrier is used
+// between the start and the end of the kernel.
+__device__ __forceinline__ void wg_bar_sync(int wg) { asm volatile("bar.sync %0, 128;" ::"r"(wg + 2) : "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
 // 128-byte swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).  High word: 8-row groups are 1024
@@ -267,15 +367,16 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   uint8_t* q_smem = smem;                                            // [q_bufs] Q operands
   uint8_t* k_smem = q_smem + p.q_bufs * q_buf_bytes;                  // [k_stages] K tiles
   uint8_t* tail = k_smem + p.k_stages * kKStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 20 barriers (28 slots reserved)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 28 * 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 28 * 8 + 4);
-  float* lse_buf = reinterpret_cast<float*>(tail + 240);              // [Ralloc] row log-sum-exps of the current pass-2 item
-  float* sm_stat = lse_buf + p.Ralloc;                            // pass 1: m[groups][Ralloc], l[groups][Ralloc]
-  float* sm_part = sm_stat + 2 * kEpiGroups * p.Ralloc;               // pass 2, several blocks per tile: [kPartSlots][groups][128] partial column sums
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);                 // 29 barriers (29 slots; the words behind them follow)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 29 * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 29 * 8 + 4);
+  float* lse_buf = reinterpret_cast<float*>(tail + 240);              // [2][Ralloc] row log-sum-exps of two pass-2 items
+  float* sm_stat = lse_buf + 2 * p.Ralloc;                            // pass 1: [2 buffers]{m[wgslots][Ralloc], l[wgslots][Ralloc]}
+  float* sm_part = sm_stat + 4 * p.wgslots * p.Ralloc;                // pass 2, several blocks per tile: [slots][groups][128] partial column sums
   const int part_slots = p.Rpad > 384 ? 4 : (p.Rpad > 128 ? 8 : 0);   // tiles in flight (see the pass-2 combine)
   int* sm_cnt = reinterpret_cast<int*>(sm_part + part_slots * kEpiGroups * 128);   // [kPartSlots][4 lane quarters] partials written
-  int* s_cu = sm_cnt + kPartSlots * 4;                                // [B+1]
+  int* sm_icnt = sm_cnt + kPartSlots * 4;                             // [2] helper warps that stored their rows of the buffer's item (+ 6 spare words)
+  int* s_cu = sm_icnt + 8;                                            // [B+1]
   int* s_prefix = s_cu + p.B + 1;                                     // [B+1]
 
   auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
@@ -284,6 +385,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   auto bar_kempty = [&](int s) { return smem_u32(&bars[8 + s]); };
   auto bar_afull = [&](int s) { return smem_u32(&bars[12 + s]); };
   auto bar_aempty = [&](int s) { return smem_u32(&bars[16 + s]); };
+  auto bar_lse_ready = [&](int s) { return smem_u32(&bars[20 + s]); };   // helper -> epilogue: lse_buf[s] holds the item's rows
+  auto bar_lse_free = [&](int s) { return smem_u32(&bars[22 + s]); };    // epilogue (16 warps) -> helper: lse_buf[s] may be rewritten
+  const uint32_t bar_drain = smem_u32(&bars[24]);
+  auto bar_stat_full = [&](int s) { return smem_u32(&bars[25 + s]); };   // epilogue (16 warps) -> helpers: the item's statistics are complete
+  auto bar_stat_free = [&](int s) { return smem_u32(&bars[27 + s]); };   // helpers -> epilogue: the statistics buffer was published                        // MMA thread: every MMA it issued has completed
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -293,16 +399,20 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     }
     for (int s = 0; s < kMaxKStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
     for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_lse_ready(s), 2); mbar_init(bar_lse_free(s), kEpiThreads / 32); }
+    mbar_init(bar_drain, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_stat_full(s), kEpiThreads / 32); mbar_init(bar_stat_free(s), 1); }
     *abort_flag = 0;
     for (int i = 0; i < kPartSlots * 4; ++i) sm_cnt[i] = 0;
+    for (int i = 0; i < 8; ++i) sm_icnt[i] = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
   }
-  if (warp == 2) {
+  if (warp == 0) {
     // sequence offsets and the per-sequence item prefix, once per CTA
     int acc = 0;
     for (int b0 = 0; b0 <= p.B; b0 += 32) {
@@ -343,123 +453,174 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   const long long npos = schedule_length(p.U, C, p.lag, p.compact != 0);
   volatile int never = 0;
 
-  if (warp == 0) {
+  unsigned long long clk0 = 0, gt0 = 0;
+  if (p.clock_out && tid == 0) { clk0 = (unsigned long long)clock64(); gt0 = global_timer_ns(); }
+
+  if (warp == kTmaWarp) {
     // ------------------------------------------------------------ TMA producer (one thread)
     if (lane == 0) {
       int stage = 0, n_item = 0;
       uint32_t phase = 0;
+      long long n_loads = 0;                          // K tiles requested so far
       bool ok = true;
+      SG_PROF_DECL(w_kempty = 0, w_qempty = 0);
       for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
         const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
         if (it.pass == 0) continue;
         const int qb = n_item % p.q_bufs;
         const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
-        ++n_item;
-        ok = mbar_wait(bar_qempty(qb), qph ^ 1u, abort_flag);
+        SG_PROF_BEGIN(tq);
+        ok = mbar_wait(bar_qempty(qb), qph ^ 1u, abort_flag, p.wait_ns, 200u);
+        SG_PROF_ADD(w_qempty, tq);
         if (!ok) break;
+        ++n_item;
         mbar_arrive_expect_tx(bar_qfull(qb), (uint32_t)(kSub * p.G * p.W * 128));
 #pragma unroll
         for (int dc = 0; dc < kSub; ++dc)
           tma_load_4d(smem_u32(q_smem + qb * q_buf_bytes + dc * q_sub_bytes), &tmap_q, bar_qfull(qb), dc * 64, it.g * p.G, 0,
                       it.l * p.B + it.b);
         for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
-          ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag);
+          SG_PROF_BEGIN(tk);
+          ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag, p.wait_ns, 200u);
+          SG_PROF_ADD(w_kempty, tk);
           if (!ok) break;
           mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
 #pragma unroll
           for (int dc = 0; dc < kSub; ++dc)
             tma_load_4d(smem_u32(k_smem + stage * kKStageBytes + dc * kKSubBytes), &tmap_k, bar_kfull(stage), dc * 64, it.g,
                         it.c0 + tile * kTileKeys, it.l);
+          ++n_loads;
           if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
         }
       }
-      // Wait until the MMAs have released every K stage and Q buffer, so that
-      // no barrier arrival and no copy of this CTA is still pending when it exits.  (On an aborted run the
-      // waits give up after their limit.)
-      for (int i = 0; i < p.k_stages; ++i) {
-        if (!mbar_wait(bar_kempty(stage), phase ^ 1u, ok ? abort_flag : &never)) break;
-        if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
-      }
-      for (int i = 0; i < p.q_bufs; ++i) {
-        const int n = n_item + i;
-        if (!mbar_wait(bar_qempty(n % p.q_bufs), (uint32_t)(((n / p.q_bufs) & 1) ^ 1), ok ? abort_flag : &never)) break;
+      SG_PROF_STORE(4, w_kempty); SG_PROF_STORE(5, w_qempty);
+      if (ok) {
+        // Wait until the MMAs have released every K stage and Q buffer: no barrier arrival and no copy of this
+        // CTA is pending when it exits.
+        for (int i = 0; i < p.k_stages; ++i) {
+          if (!mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag, p.wait_ns, 200u)) break;
+          if (++stage == p.k_stages) { stage = 0; phase ^= 1u; }
+        }
+        for (int i = 0; i < p.q_bufs; ++i) {
+          const int n = n_item + i;
+          if (!mbar_wait(bar_qempty(n % p.q_bufs), (uint32_t)(((n / p.q_bufs) & 1) ^ 1), abort_flag, p.wait_ns, 200u)) break;
+        }
+      } else {
+        // Aborted: nobody may consume what was requested, so wait (bounded, ignoring the abort flag) for the copies
+        // themselves -- the `full` barrier of every K stage and Q buffer that still has a request outstanding --
+        // before this CTA's shared memory is given up.
+        const int back = (int)(n_loads < p.k_stages ? n_loads : p.k_stages);
+        for (int i = 1; i <= back; ++i) {
+          const long long n = n_loads - i;             // the i-th last request: stage n % k_stages, use n / k_stages
+          if (!mbar_wait(bar_kfull((int)(n % p.k_stages)), (uint32_t)((n / p.k_stages) & 1), &never, p.wait_ns, 200u)) break;
+        }
+        const int qback = n_item < p.q_bufs ? n_item : p.q_bufs;
+        for (int i = 1; i <= qback; ++i) {
+          const int n = n_item - i;
+          if (!mbar_wait(bar_qfull(n % p.q_bufs), (uint32_t)((n / p.q_bufs) & 1), &never, p.wait_ns, 200u)) break;
+        }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer (one thread)
-    // Accumulator stages 0-1 feed epilogue warpgroup 0, stages 2-3 warpgroup 1; a key tile goes to the
-    // warpgroup given by the parity of the CTA's running tile count.  Each ring is consumed by one warpgroup
-    // only, so no waiter ever falls more than one mbarrier phase behind.
+    // Accumulator stage w feeds epilogue warpgroup w; block n of the CTA's running count goes to stage n mod 4.
+    // Each stage is consumed by one warpgroup only, so no waiter ever falls more than one mbarrier phase behind.
     if (lane == 0) {
       int ks = 0, n_item = 0;
-      uint32_t kph = 0, ringbits = 0, phbits = 0, tile_count = 0;   // one ring-index bit and one phase bit per warpgroup
+      uint32_t kph = 0, phbits = 0, tile_count = 0;   // phbits: one phase bit per accumulator stage
       bool ok = true;
+      SG_PROF_DECL(w_qfull = 0, w_kfull = 0, w_aempty = 0);
+      const uint32_t k_lo0 = smem_desc_lo(smem_u32(k_smem));
+      const uint32_t k_stage_lo = (uint32_t)kKStageBytes >> 4;
+      const uint32_t bar_afull0 = bar_afull(0), bar_aempty0 = bar_aempty(0);
       for (long long pos = blockIdx.x; pos < npos && ok; pos += gridDim.x) {
         const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
         if (it.pass == 0) continue;
         const int qb = n_item % p.q_bufs;
         const uint32_t qph = (uint32_t)((n_item / p.q_bufs) & 1);
         ++n_item;
-        ok = mbar_wait(bar_qfull(qb), qph, abort_flag);
+        SG_PROF_BEGIN(tq);
+        ok = mbar_wait(bar_qfull(qb), qph, abort_flag, p.wait_ns, 0u);
+        SG_PROF_ADD(w_qfull, tq);
         if (!ok) break;
         tc_fence_after();
+        // per-item constants of the issue loop
         const bool pass1 = it.pass == 1;
         const int nblk = pass1 ? (p.R + 127) / 128 : (p.Rpad + 127) / 128;
-        const uint32_t q_addr = smem_u32(q_smem + qb * q_buf_bytes);
+        const uint32_t q_lo0 = smem_desc_lo(smem_u32(q_smem + qb * q_buf_bytes));
+        const uint32_t q_blk_lo = (128u * 128u) >> 4;                      // next row block of the Q operand
+        const uint32_t a_sub = (uint32_t)(pass1 ? q_sub_bytes : kKSubBytes) >> 4;
+        const uint32_t b_sub = (uint32_t)(pass1 ? kKSubBytes : q_sub_bytes) >> 4;
+        const uint32_t idesc_full = make_idesc(128, 128);
+        const uint32_t idesc_last = pass1 ? idesc_full : make_idesc(128, p.Rpad - (nblk - 1) * 128);
         for (int tile = it.tile_beg; tile < it.tile_end && ok; ++tile) {
-          ok = mbar_wait(bar_kfull(ks), kph, abort_flag);
+          SG_PROF_BEGIN(tk);
+          if (!mbar_test(bar_kfull(ks), kph)) ok = mbar_wait(bar_kfull(ks), kph, abort_flag, p.wait_ns, 0u);
+          SG_PROF_ADD(w_kfull, tk);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(k_smem + ks * kKStageBytes);
-          const bool blockwise = nblk > 1;                 // several blocks per key tile: deal blocks, not tiles
-          uint32_t wgsel = blockwise ? 0u : (tile_count++) % kEpiGroups;
-          for (int blk = 0; blk < nblk && ok; ++blk) {
-            if (blockwise) wgsel = (tile_count++) % kEpiGroups;
-            const uint32_t ridx = kRing == 2 ? ((ringbits >> wgsel) & 1u) : 0u;
-            const int as = (int)(wgsel * kRing + ridx);
-            ok = mbar_wait(bar_aempty(as), ((phbits >> wgsel) & 1u) ^ 1u, abort_flag);
+          const uint32_t k_lo = k_lo0 + (uint32_t)ks * k_stage_lo;
+          uint32_t q_lo = q_lo0;
+          for (int blk = 0; blk < nblk; ++blk, q_lo += q_blk_lo) {
+            const uint32_t as = (tile_count++) % kEpiGroups;               // blocks go to the warpgroups in rotation
+            const uint32_t par = ((phbits >> as) & 1u) ^ 1u;
+            SG_PROF_EVENT(8, tile_count - 1);
+            SG_PROF_BEGIN(ta);
+            const bool fast = mbar_test(bar_aempty0 + as * 8u, par);
+            SG_PROF_EVENT(9, tile_count - 1);
+            if (!fast) ok = mbar_wait(bar_aempty0 + as * 8u, par, abort_flag, p.wait_ns, 0u);
+            SG_PROF_ADD(w_aempty, ta);
+            SG_PROF_EVENT(0, tile_count - 1);
             if (!ok) break;
             tc_fence_after();
-            const int ncols = pass1 ? 128 : min(128, p.Rpad - blk * 128);
-            const uint32_t idesc = make_idesc(128, ncols);
-            const uint32_t d_tmem = tmem_base + (uint32_t)(as * 128);
-            const uint32_t q_lo = smem_desc_lo(q_addr + blk * (128 * 128));
-            const uint32_t k_lo = smem_desc_lo(k_addr);
-            const uint32_t a_lo = pass1 ? q_lo : k_lo, b_lo = pass1 ? k_lo : q_lo;
-            const uint32_t a_sub = (uint32_t)(pass1 ? q_sub_bytes : kKSubBytes) >> 4;
-            const uint32_t b_sub = (uint32_t)(pass1 ? kKSubBytes : q_sub_bytes) >> 4;
-            umma_bf16<false>(d_tmem, a_lo, b_lo, kSmemDescHi, idesc);
-#pragma unroll
-            for (int i = 1; i < 4 * kSub; ++i) {
-              const uint32_t dc = (uint32_t)(i >> 2), kk = (uint32_t)(i & 3);
-              umma_bf16<true>(d_tmem, a_lo + dc * a_sub + kk * 2, b_lo + dc * b_sub + kk * 2, kSmemDescHi, idesc);
-            }
-            umma_commit(bar_afull(as));
-            if (kRing == 2) { ringbits ^= 1u << wgsel; if (ridx == 1u) phbits ^= 1u << wgsel; }
-            else phbits ^= 1u << wgsel;
+            umma_block<4 * kSub>(tmem_base + as * 128u, pass1 ? q_lo : k_lo, pass1 ? k_lo : q_lo, a_sub, b_sub, kSmemDescHi,
+                                 blk == nblk - 1 ? idesc_last : idesc_full);
+            SG_PROF_EVENT(7, tile_count - 1);
+            umma_commit(bar_afull0 + as * 8u);
+            SG_PROF_EVENT(1, tile_count - 1);
+            phbits ^= 1u << as;
           }
           if (ok) umma_commit(bar_kempty(ks));
           if (++ks == p.k_stages) { ks = 0; kph ^= 1u; }
         }
         if (ok) umma_commit(bar_qempty(qb));
       }
+      // Every MMA this thread issued has completed before the CTA frees its tensor memory, also on an aborted run
+      // (the commit arrives when all earlier MMAs are done; the wait ignores the abort flag and is bounded).
+      SG_PROF_STORE(6, w_qfull); SG_PROF_STORE(7, w_kfull); SG_PROF_STORE(8, w_aempty);
+      umma_commit(bar_drain);
+      mbar_wait(bar_drain, 0u, &never, p.wait_ns, 0u);
     }
-  } else {
+  } else if (warp < kTmaWarp) {
     // ------------------------------------------------------------ epilogue warps
-    // Warpgroups of four warps; each owns whole key tiles (every kEpiGroups-th of the CTA's running count), so a
-    // thread sees all 128 accumulator columns of its TMEM lane and no per-tile exchange between warps is needed.
-    const int etid = tid - 64;
-    const int wg = (warp - 2) >> 2;
+    // Four warpgroups of four warps; each owns one accumulator stage and every fourth block (a key tile, or one
+    // row block of a key tile) of the CTA's running block count.  A thread sees all 128 accumulator columns of
+    // its TMEM lane.  The warpgroups never meet at a CTA-wide barrier: each walks the CTA's items on its own,
+    // publishes its own pass-1 statistics and waits only for accumulators and (pass 2) for the helper warp's
+    // log-sum-exps, so the others keep the SFU busy while one of them is between items.
+    const int wg = warp >> 2;
+    const int wg_tid = tid & 127;
     const int lane_grp = warp & 3;                     // TMEM lane quarter this warp may access
     const int row_in_tile = lane_grp * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
-    int ring = 0;                                      // this warpgroup's ring of two accumulator stages
+    const int as = wg;                                 // this warpgroup's accumulator stage
+    const uint32_t t_acc = t_lane + (uint32_t)(as * 128);
+    const int wgslot = p.wgslots == 4 ? wg : 0;
     uint32_t aph = 0, tile_count = 0;
+    int n_p2 = 0;                                      // pass-2 items seen so far (selects the lse buffer)
+    int n_p1 = 0;                                      // pass-1 items seen so far (selects the statistics buffer)
     bool ok = true;
-    auto next_stage = [&]() {
-      if (++ring == kRing) { ring = 0; aph ^= 1u; }
+    SG_PROF_DECL(w_afull = 0, w_lse = 0, w_pub = 0, n_blocks = 0);
+    // Releases the accumulator: called right after the block's last TMEM load has completed, before the
+    // arithmetic on those columns, so the MMAs of this warpgroup's next block overlap it.
+    auto release_acc = [&]() {
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_aempty(as));
+      aph ^= 1u;
+      if (lane == 0) SG_PROF_EVENT(3 + lane_grp, tile_count - 1);
     };
-    for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every warp meets the named barriers
+    for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every thread meets its warpgroup's barriers
       const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
       if (it.pass == 0) continue;
       const int N = it.N;
@@ -468,50 +629,79 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
 
       if (it.pass == 1) {
         const int nblk = (p.R + 127) / 128;
-        float* sm_m = sm_stat;                         // [groups][Ralloc], one copy per warpgroup
-        float* sm_l = sm_stat + kEpiGroups * p.Ralloc;
-        for (int r = etid; r < kEpiGroups * p.Ralloc; r += kEpiThreads) { sm_m[r] = -INFINITY; sm_l[r] = 0.f; }
-        epi_bar_sync();
+        const bool blockwise = nblk > 1;
+        const uint32_t n_item0 = tile_count;           // running block count at the start of the item
+        // Running statistics live in one of two shared-memory buffers (alternating pass-1 items, because the
+        // warpgroups drift apart by up to an item).  The buffer's previous item must have been merged and published
+        // by the helper warps (practically always true already; the wait is bounded).
+        const int sbuf = n_p1 & 1, suse = n_p1 >> 1;
+        ++n_p1;
+        if (ok && suse > 0) ok = mbar_wait(bar_stat_free(sbuf), (uint32_t)((suse - 1) & 1), abort_flag, p.wait_ns, 32u);
+        float* sm_m = sm_stat + (size_t)(sbuf * 2 * p.wgslots + wgslot) * p.Ralloc;   // this warpgroup's slot: max ...
+        float* sm_l = sm_m + p.wgslots * p.Ralloc;                                     // ... and sum of exp2
+        // Slot (wgslot, blk*128 + row_in_tile) is only ever touched by this thread during the item, so the running
+        // statistics need no barrier: with one slot per warpgroup every block's rows are initialised, with a shared
+        // slot (the number of row blocks is a multiple of four, so a row block always meets the same warpgroup)
+        // only the owned ones.
+        for (int blk = 0; blk < nblk; ++blk)
+          if (p.wgslots == 4 || ((n_item0 + (uint32_t)blk) % kEpiGroups) == (uint32_t)wg) {
+            sm_m[blk * 128 + row_in_tile] = -INFINITY;
+            sm_l[blk * 128 + row_in_tile] = 0.f;
+          }
         for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
-          const bool blockwise = nblk > 1;
           if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t0 = tile * kTileKeys;
           const bool all_visible = t0 + kTileKeys - 1 <= first_win;
           for (int blk = 0; blk < nblk; ++blk) {
             if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
-            const int as = wg * kRing + ring;
-            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            SG_PROF_BEGIN(ta);
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
+            SG_PROF_ADD(w_afull, ta);
+            SG_PROF_INC(n_blocks);
+            if (wg_tid == 0) SG_PROF_EVENT(2, tile_count - 1);
             if (!ok) continue;
             tc_fence_after();
             const int r = blk * 128 + row_in_tile;
             const bool row_ok = r < p.R && (r / p.G) < Weff;
             const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
-            float m = sm_m[wg * p.Ralloc + r], lsum = sm_l[wg * p.Ralloc + r];
-            const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
-            uint32_t cur[32];                            // (four warps per scheduler hide the TMEM load latency)
-#pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-              const int col0 = j * 32;
-              tmem_ld32(cur, t_blk + (uint32_t)col0);
+            float m = sm_m[r], lsum = sm_l[r];
+            // one 32-column chunk of this thread's row: online (max, sum of exp2) in the log2 domain
+            auto chunk = [&](const uint32_t (&cur)[32], const int col0) {
               if (all_visible && row_ok) {
-                float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
-                float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
-#pragma unroll
-                for (int c = 4; c < 32; c += 4) {
-                  mx0 = fmaxf(mx0, __uint_as_float(cur[c]));     mx1 = fmaxf(mx1, __uint_as_float(cur[c + 1]));
-                  mx2 = fmaxf(mx2, __uint_as_float(cur[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(cur[c + 3]));
-                }
-                const float mn = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                // The running reference m need not be the row maximum: fp32 keeps its relative precision for any
+                // exponent, so the sum of exp2(x - m) is as accurate with a stale (lower) m as with the true maximum,
+                // as long as nothing overflows.  The chunk is therefore summed against the current m first (no
+                // maximum over its 32 values); only if the sum leaves the safe range -- a value more than ~60 binary
+                // orders above m, or m still -inf at the start of an item -- is the maximum taken and the chunk redone.
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 32; c += 4) {
-                  s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn));
-                  s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -mn));
-                  s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -mn));
-                  s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -mn));
+                  s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -m));
+                  s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -m));
+                  s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -m));
+                  s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -m));
                 }
-                lsum = lsum * exp2f(m - mn) + ((s0 + s1) + (s2 + s3));
-                m = mn;
+                const float s = (s0 + s1) + (s2 + s3);
+                if (s < 0x1p60f) {
+                  lsum += s;
+                } else {
+                  float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
+                  float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
+#pragma unroll
+                  for (int c = 4; c < 32; c += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(cur[c]));     mx1 = fmaxf(mx1, __uint_as_float(cur[c + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(cur[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(cur[c + 3]));
+                  }
+                  const float mn = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                  float r0 = 0.f, r1 = 0.f;
+#pragma unroll
+                  for (int c = 0; c < 32; c += 2) {
+                    r0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn));
+                    r1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -mn));
+                  }
+                  lsum = lsum * exp2f(m - mn) + (r0 + r1);
+                  m = mn;
+                }
               } else if (col0 <= cmax) {
                 float mx = -INFINITY;
 #pragma unroll
@@ -524,71 +714,46 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 lsum = lsum * exp2f(m - mn) + s;
                 m = mn;
               }
+            };
+            uint32_t cur[32];
+#ifdef SG_SCORE_PROFILE
+            if (p.debug_mode == 1) { release_acc(); continue; }
+#endif
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+              tmem_ld_wait(cur);
+              if (j == 3) release_acc();
+#ifdef SG_SCORE_PROFILE
+              if (p.debug_mode == 2) continue;
+#endif
+              chunk(cur, j * 32);
             }
-            sm_m[wg * p.Ralloc + r] = m;
-            sm_l[wg * p.Ralloc + r] = lsum;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_aempty(as));
-            next_stage();
+            sm_m[r] = m;
+            sm_l[r] = lsum;
           }
         }
-        epi_bar_sync();
-        const size_t slot = ((size_t)it.unit * p.max_items + it.item_in_unit) * p.Ralloc;
-        for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
-          float M = -INFINITY;
-#pragma unroll
-          for (int w = 0; w < kEpiGroups; ++w) M = fmaxf(M, sm_m[w * p.Ralloc + r]);
-          const float Mu = M == -INFINITY ? 0.f : M;
-          float L = 0.f;
-#pragma unroll
-          for (int w = 0; w < kEpiGroups; ++w) L += sm_l[w * p.Ralloc + r] * exp2f(sm_m[w * p.Ralloc + r] - Mu);
-          p.part_m[slot + r] = M;
-          p.part_l[slot + r] = L;
-        }
-        epi_bar_sync();                                // every thread's statistics are written (CTA-wide order) ...
-        if (etid == 0 && ok && !*abort_flag) {
-          __threadfence();                             // ... made visible GPU-wide by one cumulative fence ...
-          atomicAdd(p.p1_done + it.unit, 1);           // ... before the item is counted as done
-        }
+        // End of the item for this warp: its rows' statistics are complete in shared memory.  The helper warps merge
+        // the warpgroups' slots, publish the item and count it as done for its unit, off this warp's path.
+        SG_PROF_BEGIN(tp);
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(bar_stat_full(sbuf));
+        SG_PROF_ADD(w_pub, tp);
       } else {
         const int nblk = (p.Rpad + 127) / 128;
-        float* lse2 = lse_buf;                         // [Ralloc] row log-sum-exps (log2 domain) of (unit, b)
-        // Wait (bounded) until every pass-1 item of this unit has published its row statistics.
-        if (etid == 0 && ok) {
-          uint64_t t0 = 0;
-          for (uint32_t spin = 0; ld_acquire_gpu(p.p1_done + it.unit) < C; ++spin) {
-            if (*abort_flag) break;
-            if ((spin & 63u) == 63u) {
-              const uint64_t now = global_timer_ns();
-              if (t0 == 0) t0 = now;
-              else if (now - t0 > 2000000000ull) { *abort_flag = 1; break; }
-            }
-            __nanosleep(64);
-          }
-        }
-        epi_bar_sync();
-        if (*abort_flag) ok = false;
-        {
-          const size_t part_base = ((size_t)it.unit * p.max_items + it.first_item_b) * p.Ralloc;
-          for (int r = etid; r < p.Ralloc; r += kEpiThreads) {
-            float val = INFINITY;                      // rows outside the window: exp2(x - inf) = 0
-            if (ok && r < p.R && (r / p.G) < Weff) {
-              float M = -INFINITY;
-              for (int c = 0; c < it.nch_b; ++c) M = fmaxf(M, __ldcg(p.part_m + part_base + (size_t)c * p.Ralloc + r));
-              float L = 0.f;
-              for (int c = 0; c < it.nch_b; ++c) {
-                const size_t o = part_base + (size_t)c * p.Ralloc + r;
-                L += __ldcg(p.part_l + o) * exp2f(__ldcg(p.part_m + o) - M);
-              }
-              val = M + log2f(L);
-            }
-            lse2[r] = val;
-          }
-        }
-        epi_bar_sync();
+        const bool blockwise = nblk > 1;
+        // The helper warp has merged the unit's pass-1 statistics into this item's row log-sum-exps (it waited for
+        // the unit's counter); two buffers, so it works on the next pass-2 item while this one runs.  Every warp
+        // waits here, also one that gets no block of the item: passing this point proves that the buffer's previous
+        // use was released by all sixteen warps, which keeps the arrivals below in step with the barrier's phases.
+        const int lbuf = n_p2 & 1;
+        const uint32_t lph = (uint32_t)((n_p2 >> 1) & 1);
+        ++n_p2;
+        SG_PROF_BEGIN(tl);
+        if (ok) ok = mbar_wait(bar_lse_ready(lbuf), lph, abort_flag, p.wait_ns, 32u);
+        SG_PROF_ADD(w_lse, tl);
+        const float* lse2 = lse_buf + lbuf * p.Ralloc;   // [Ralloc] row log-sum-exps (log2 domain) of (unit, b)
         for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
-          const bool blockwise = nblk > 1;
           if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t = tile * kTileKeys + row_in_tile;  // this thread's key
           const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
@@ -599,41 +764,49 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           for (int blk = 0; blk < nblk; ++blk) {
             if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
             mine = true;
-            const int as = wg * kRing + ring;
-            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag);
+            SG_PROF_BEGIN(ta);
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
+            SG_PROF_ADD(w_afull, ta);
+            SG_PROF_INC(n_blocks);
+            if (wg_tid == 0) SG_PROF_EVENT(2, tile_count - 1);
             if (!ok) continue;
             tc_fence_after();
             const int ncols = min(128, p.Rpad - blk * 128);
-            const uint32_t t_blk = t_lane + (uint32_t)(as * 128);
-            uint32_t cur[32];
-#pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-              const int col0 = j * 32;
-              if (col0 < ncols) {
-                tmem_ld32(cur, t_blk + (uint32_t)col0);
-                const float* ls = lse2 + blk * 128 + col0;
-                if (all_visible && col0 + 32 <= ncols) {
+            const int nchk = (ncols + 31) >> 5;          // 32-column chunks of this block (warp-uniform)
+            // one 32-column chunk of this thread's key: add exp2(s*c - lse_r) over the visible query rows
+            auto chunk = [&](const uint32_t (&cur)[32], const int col0) {
+              const float* ls = lse2 + blk * 128 + col0;
+              if (all_visible && col0 + 32 <= ncols) {
 #pragma unroll
-                  for (int c = 0; c < 32; c += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                    a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
-                    a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
-                    a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
-                    a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
-                  }
-                } else {
+                for (int c = 0; c < 32; c += 4) {
+                  const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                  a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
+                  a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
+                  a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
+                  a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
+                }
+              } else {
 #pragma unroll
-                  for (int c = 0; c < 32; ++c) {
-                    const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
-                    a0 += vis ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -ls[c])) : 0.f;
-                  }
+                for (int c = 0; c < 32; ++c) {
+                  const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
+                  a0 += vis ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -ls[c])) : 0.f;
                 }
               }
+            };
+            uint32_t cur[32];
+#ifdef SG_SCORE_PROFILE
+            if (p.debug_mode == 1) { release_acc(); continue; }
+#endif
+#pragma unroll 1
+            for (int j = 0; j < nchk; ++j) {
+              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+              tmem_ld_wait(cur);
+              if (j == nchk - 1) release_acc();
+#ifdef SG_SCORE_PROFILE
+              if (p.debug_mode == 2) continue;
+#endif
+              chunk(cur, j * 32);
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_aempty(as));
-            next_stage();
           }
           float total = (a0 + a1) + (a2 + a3);
           if (blockwise) {
@@ -662,19 +835,155 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           }
           if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
         }
-        epi_bar_sync();                                // lse2 is rewritten by the next pass-2 item
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(bar_lse_free(lbuf));        // this warp no longer reads lse_buf[lbuf]
       }
     }
+#ifdef SG_SCORE_PROFILE
+    if (wg_tid == 0) { SG_PROF_STORE(9 + wg * 4, w_afull); SG_PROF_STORE(10 + wg * 4, w_lse); SG_PROF_STORE(11 + wg * 4, w_pub); SG_PROF_STORE(12 + wg * 4, n_blocks); }
+#endif
+  } else if (warp >= kHelperWarp) {
+    // ------------------------------------------------------------ helper warps (two: each handles half of the rows)
+    // Everything at an item boundary that is not arithmetic on scores runs here, off the epilogue's path:
+    //   publish(k), k-th pass-1 item of this CTA: when all sixteen epilogue warps have left their statistics in shared
+    //     memory, merge the warpgroups' slots per row, store one (max, sum) pair per row for the item, count the item
+    //     as done for its unit (stores ordered before the count by a fence), and hand the buffer back;
+    //   lse(j), j-th pass-2 item: when all pass-1 items of the unit are counted (bounded wait), merge the chunks' pairs
+    //     of the item's sequence into the rows' log-sum-exps for the epilogue; this runs one pass-2 item ahead of it.
+    // The two sequences advance independently and neither ever blocks: a task is taken only when a test shows that it
+    // can run, so a publication this CTA owes can never be held up behind a count some other CTA still owes.
+    const int hw = warp - kHelperWarp;
+    long long pos1 = blockIdx.x, pos2 = blockIdx.x;      // schedule cursors of the next pass-1 / pass-2 item
+    int k1 = 0, j2 = 0;
+    ScoreItem it1, it2;
+    it1.pass = it2.pass = 0;
+    auto next_item = [&](long long& pos, ScoreItem& it, int pass) {   // advance to the next item of `pass` (it.pass = 0: none left)
+      for (; pos < npos; pos += gridDim.x) {
+        it = decode_position(p, pos, s_cu, s_prefix);
+        if (it.pass == pass) { pos += gridDim.x; return; }
+      }
+      it.pass = 0;
+    };
+    next_item(pos1, it1, 1);
+    next_item(pos2, it2, 2);
+    uint64_t idle_since = 0;
+    uint32_t idle_iters = 0;
+    SG_PROF_DECL(h_free = 0, h_cnt = 0, h_merge = 0);
+    while (it1.pass != 0 || it2.pass != 0) {
+      bool progressed = false;
+      if (it1.pass != 0 && mbar_test(bar_stat_full(k1 & 1), (uint32_t)((k1 >> 1) & 1))) {
+        SG_PROF_BEGIN(th0);
+        const int sbuf = k1 & 1;
+        const float* bm = sm_stat + (size_t)(sbuf * 2 * p.wgslots) * p.Ralloc;
+        const float* bl = bm + p.wgslots * p.Ralloc;
+        const size_t slot = ((size_t)it1.unit * p.max_items + it1.item_in_unit) * p.Ralloc;
+        for (int r = hw * 32 + lane; r < p.Ralloc; r += 64) {
+          float M = bm[r];
+          for (int w = 1; w < p.wgslots; ++w) M = fmaxf(M, bm[w * p.Ralloc + r]);
+          const float Mu = M == -INFINITY ? 0.f : M;
+          float L = 0.f;
+          for (int w = 0; w < p.wgslots; ++w) L += bl[w * p.Ralloc + r] * exp2f(bm[w * p.Ralloc + r] - Mu);
+          p.part[slot + r] = make_float2(M, L);
+        }
+        __threadfence();                               // this warp's stores, GPU-wide, before it reports in
+        __syncwarp();
+        int second = 0;
+        if (lane == 0) second = atomicAdd(&sm_icnt[sbuf], 1);
+        second = __shfl_sync(0xffffffffu, second, 0);
+        if (second == 1 && lane == 0) {                  // both helper warps have stored their rows
+          sm_icnt[sbuf] = 0;
+          __threadfence();
+          if (!*abort_flag && it1.unit != p.withhold_unit) atomicAdd(p.p1_done + it1.unit, 1);
+          mbar_arrive(bar_stat_free(sbuf));
+        }
+        ++k1;
+        next_item(pos1, it1, 1);
+        progressed = true;
+        SG_PROF_ADD(h_free, th0);
+      }
+      if (it2.pass != 0) {
+        const int lbuf = j2 & 1, use = j2 >> 1;
+        bool can = use == 0 || mbar_test(bar_lse_free(lbuf), (uint32_t)((use - 1) & 1));
+        if (can) {
+          int cnt = 0;
+          if (lane == 0) cnt = ld_acquire_gpu(p.p1_done + it2.unit);
+          cnt = __shfl_sync(0xffffffffu, cnt, 0);
+          can = cnt >= C;
+        }
+        if (can) {
+          SG_PROF_BEGIN(th2);
+          __syncwarp();
+          __threadfence();                             // the other lanes' loads follow lane 0's acquire
+          float* lse2 = lse_buf + lbuf * p.Ralloc;
+          const int Weff = min(p.W, it2.N);
+          const size_t part_base = ((size_t)it2.unit * p.max_items + it2.first_item_b) * p.Ralloc;
+          const int nparts = it2.nch_b;
+          // a lane merges two neighbouring rows at a time (one 16-byte load per chunk), eight loads in flight
+          for (int r = 2 * (hw * 32 + lane); r < p.Ralloc; r += 128) {
+            float M0 = -INFINITY, L0 = 0.f, M1 = -INFINITY, L1 = 0.f;
+            for (int c0 = 0; c0 < nparts; c0 += 8) {
+              float4 v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                v[i] = c0 + i < nparts ? __ldcg(reinterpret_cast<const float4*>(p.part + part_base + (size_t)(c0 + i) * p.Ralloc + r))
+                                       : make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+              float m0 = v[0].x, m1 = v[0].z;
+#pragma unroll
+              for (int i = 1; i < 8; ++i) { m0 = fmaxf(m0, v[i].x); m1 = fmaxf(m1, v[i].z); }
+              if (m0 != -INFINITY) {                   // else nothing of row r is visible in these chunks
+                const float Mn = fmaxf(M0, m0);
+                float acc = L0 * exp2f(M0 - Mn);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc += v[i].y * exp2f(v[i].x - Mn);   // a (-inf, 0) pair adds 0
+                M0 = Mn; L0 = acc;
+              }
+              if (m1 != -INFINITY) {
+                const float Mn = fmaxf(M1, m1);
+                float acc = L1 * exp2f(M1 - Mn);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc += v[i].w * exp2f(v[i].z - Mn);
+                M1 = Mn; L1 = acc;
+              }
+            }
+            // rows outside the window get +inf: exp2(x - inf) = 0
+            lse2[r] = (r < p.R && (r / p.G) < Weff) ? M0 + log2f(L0) : INFINITY;
+            lse2[r + 1] = (r + 1 < p.R && ((r + 1) / p.G) < Weff) ? M1 + log2f(L1) : INFINITY;
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_lse_ready(lbuf));
+          ++j2;
+          next_item(pos2, it2, 2);
+          progressed = true;
+          SG_PROF_ADD(h_merge, th2);
+        }
+      }
+      if (progressed) { idle_since = 0; idle_iters = 0; continue; }
+      // nothing could run: sleep a little; every 16th idle round look at the abort flag and the clock (bounded wait)
+      __nanosleep(200);
+      if ((++idle_iters & 15u) == 0u) {
+        if (*abort_flag) break;
+        const uint64_t now = global_timer_ns();
+        if (idle_since == 0) idle_since = now;
+        else if (now - idle_since > 2ull * p.wait_ns) { *abort_flag = 1; break; }
+      }
+    }
+#ifdef SG_SCORE_PROFILE
+    if (warp == kHelperWarp && lane == 0) { SG_PROF_STORE(25, h_free); SG_PROF_STORE(26, h_cnt); SG_PROF_STORE(27, h_merge); }
+#endif
   }
 
   // ---------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
   if (tid == 0 && *abort_flag) raise(p.dev_status, SG_ERR_TIMEOUT);
+  if (p.clock_out && tid == 0) {
+    unsigned long long* o = p.clock_out + kClockWords * (size_t)blockIdx.x;
+    o[0] = clk0; o[1] = (unsigned long long)clock64(); o[2] = gt0; o[3] = global_timer_ns();
+  }
 }
 
 // ---------------------------------------------------------------- host side
@@ -693,8 +1002,13 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Testing hooks (sg_testing_score_fault, sg_testing_score_clock): process-wide, off by default.
+std::atomic<int> g_test_withhold_unit{-1};
+std::atomic<int> g_test_wait_limit_ms{0};
+std::atomic<unsigned long long*> g_test_clock_out{nullptr};
+
 struct ScorePlan {
-  int R, Rpad, Ralloc, k_stages, q_bufs, tiles_per_chunk, max_items, smem_bytes, U, lag;
+  int R, Rpad, Ralloc, k_stages, q_bufs, tiles_per_chunk, max_items, smem_bytes, U, lag, wgslots;
   size_t counter_bytes, workspace_bytes;
   bool ok;
 };
@@ -709,7 +1023,11 @@ ScorePlan plan_score(const sg_shape* s) {
   const int q_bytes = pl.Ralloc * D * 2;
   const int k_stage = kTileKeys * D * 2;
   const int part_slots = pl.Rpad > 384 ? 4 : (pl.Rpad > 128 ? 8 : 0);
-  const int tail = (240 + (1 + 2 * kEpiGroups) * pl.Ralloc * 4 + part_slots * kEpiGroups * 128 * 4 + kPartSlots * 4 * 4 + 2 * (s->batch + 1) * 4 + 15) & ~15;
+  // Row blocks are dealt to the four epilogue warpgroups in rotation.  When their number is a multiple of four a
+  // row block always meets the same warpgroup, so one statistics slot per item suffices; otherwise every
+  // warpgroup keeps (and publishes) its own.
+  pl.wgslots = ((pl.Ralloc / 128) % kEpiGroups == 0) ? 1 : kEpiGroups;
+  const int tail = (240 + (2 + 4 * pl.wgslots) * pl.Ralloc * 4 + part_slots * kEpiGroups * 128 * 4 + kPartSlots * 4 * 4 + 32 + 2 * (s->batch + 1) * 4 + 15) & ~15;
   const int avail = kSmemLimit - 1024 - tail;
   // Two Q buffers let the next item's queries load while the current item computes; fall back to one
   // when that would leave fewer than three K stages.
@@ -728,6 +1046,7 @@ ScorePlan plan_score(const sg_shape* s) {
   const int64_t tiles_per_unit = (int64_t)s->total_tokens / kTileKeys + s->batch;
   int tpc = pl.R >= 256 ? 32 : 16;
   while (tpc > 4 && (tiles_per_unit / tpc + s->batch) * pl.U < 6 * kNumSMs) tpc /= 2;
+  if (getenv("SG_SCORE_TPC")) tpc = atoi(getenv("SG_SCORE_TPC"));   // EXPERIMENT
   pl.tiles_per_chunk = tpc;
   pl.max_items = (int)(tiles_per_unit / tpc + s->batch + 1);
   // Pass 2 of a unit trails its pass 1 by `lag` units.  The lag must span more schedule positions than there
@@ -735,7 +1054,8 @@ ScorePlan plan_score(const sg_shape* s) {
   // items they wait for and stall; beyond that it is kept as small as possible so that the unit's keys are
   // still in L2 for the second read.
   const int64_t c_est = (tiles_per_unit - s->batch) / tpc + 1;
-  int64_t lag = (5 * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
+  static const int lag_num = getenv("SG_SCORE_LAGNUM") ? atoi(getenv("SG_SCORE_LAGNUM")) : 14;   // EXPERIMENT
+  int64_t lag = (lag_num * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
   if (2 * lag > pl.U) lag = pl.U;     // few units: all pass-1 items first, then all pass-2 items
   pl.lag = (int)lag;
   pl.counter_bytes = ((size_t)pl.U * sizeof(int) + 255) & ~(size_t)255;
@@ -784,6 +1104,24 @@ size_t score_workspace_bytes(const sg_shape* s) {
 }
 
 }  // namespace sg
+
+extern "C" void sg_testing_score_fault(int32_t withhold_unit, int32_t wait_limit_ms) {
+  sg::g_test_withhold_unit.store(withhold_unit, std::memory_order_relaxed);
+  sg::g_test_wait_limit_ms.store(wait_limit_ms, std::memory_order_relaxed);
+}
+
+extern "C" void sg_testing_score_clock(void* dev_buffer) {
+  sg::g_test_clock_out.store(static_cast<unsigned long long*>(dev_buffer), std::memory_order_relaxed);
+}
+
+extern "C" int32_t sg_testing_score_grid(const sg_shape* shape) {
+  using namespace sg;
+  if (check_shape(shape, true) != SG_OK) return 0;
+  const ScorePlan pl = plan_score(shape);
+  if (!pl.ok) return 0;
+  const long long max_pos = (long long)(pl.U + pl.lag) * 2 * pl.max_items;
+  return (int32_t)(max_pos < kNumSMs ? max_pos : kNumSMs);
+}
 
 extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const void* k_cache, float* importance,
                               void* workspace, size_t workspace_bytes, int32_t* dev_status, void* stream) {
@@ -836,8 +1174,7 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   p.cu = shape->cu_seqlens;
   p.importance = importance;
   p.p1_done = static_cast<int*>(workspace);
-  p.part_m = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
-  p.part_l = p.part_m + (size_t)pl.U * pl.max_items * pl.Ralloc;
+  p.part = reinterpret_cast<float2*>(static_cast<uint8_t*>(workspace) + pl.counter_bytes);
   p.dev_status = dev_status;
   p.T = shape->total_tokens;
   p.B = shape->batch;
@@ -853,6 +1190,12 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   p.max_items = pl.max_items;
   p.k_stages = pl.k_stages;
   p.q_bufs = pl.q_bufs;
+  p.wgslots = pl.wgslots;
+  p.debug_mode = getenv("SG_SCORE_DEBUG") ? atoi(getenv("SG_SCORE_DEBUG")) : 0;   // EXPERIMENT
+  p.withhold_unit = g_test_withhold_unit.load(std::memory_order_relaxed);
+  const int limit_ms = g_test_wait_limit_ms.load(std::memory_order_relaxed);
+  p.wait_ns = limit_ms > 0 ? (uint32_t)limit_ms * 1000000u : 1000000000u;
+  p.clock_out = g_test_clock_out.load(std::memory_order_relaxed);
   p.scale_log2 = kLog2e / sqrtf((float)D);
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -881,7 +1224,9 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
 // The row statistics that pass 1 hands to pass 2 normally live in a caller-provided workspace.
 // Here they live in a fixed array that is part of the library image, so the caller needs no
 // allocator at all.  The array is shared by every call on a device and keeps the previous call's
-// contents; nothing in it has to start at zero, because pass 1 writes every slot that pass 2 reads.
+// contents.  The per-unit completion counters at its start must be zero when the kernel begins: the
+// call clears them with a memset on `stream`, exactly as sg_score does for a caller's workspace.
+// Every other word is written by pass 1 before pass 2 reads it.
 namespace sg {
 namespace {
 static __device__ __align__(256) unsigned char g_score_static_scratch[SG_SCORE_STATIC_SCRATCH_BYTES];
@@ -893,6 +1238,8 @@ extern "C" sg_status sg_score_static(const sg_shape* shape, const void* q_win, c
   using namespace sg;
   sg_status st = check_shape(shape, true);
   if (st != SG_OK) return st;
+  if (shape->total_tokens == 0) return SG_OK;
+  if (!plan_score(shape).ok) return SG_ERR_UNSUPPORTED;      // same answer as sg_score for shapes no kernel covers
   if (score_workspace_bytes(shape) > (size_t)SG_SCORE_STATIC_SCRATCH_BYTES) return SG_ERR_WORKSPACE;
   // In host code the array's name is only a handle; the device address has to be asked for, once per
   // device, with that device current.
