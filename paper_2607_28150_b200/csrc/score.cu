@@ -12,23 +12,24 @@
 //          each epilogue thread owns one key (one TMEM lane) and adds exp2(s*c - lse_r) over the
 //          query-row columns; lse_r is a per-column constant read from shared memory.
 //
-// One persistent kernel runs both passes: warp 0 feeds Q and 128-key K tiles with TMA into
-// 128-byte-swizzled shared memory, warp 1 issues tcgen05.mma into four 128-column TMEM accumulator
-// stages (one per epilogue warpgroup), the epilogue warps (four warpgroups, each owning every fourth key tile) drain them with pipelined
-// tcgen05.ld.  The score matrix never leaves the SM.  Work items (a pass, a layer/KV head, a chunk of
-// key tiles of one sequence) are laid out so that pass 2 of a (layer, KV head) unit follows its pass 1
-// by a lag of a few units: close enough that the unit's keys are still in L2 for the second read
-// (K crosses HBM once), far enough that the statistics pass 2 needs are already published.  Pass 1
-// items publish per-chunk row statistics to a small workspace and bump a per-unit counter; pass 2 items
-// wait (bounded) on that counter and merge the chunks' statistics into the rows' log-sum-exps.  A pass-2 item only depends on items at smaller schedule positions and
-// pass-1 items never wait, so the schedule cannot deadlock for any grid size.
+// One persistent kernel runs both passes: one warp feeds Q and 128-key K tiles with TMA into 128-byte-swizzled
+// shared memory, one thread issues tcgen05.mma into four 128-column TMEM accumulator stages (one per epilogue
+// warpgroup), sixteen epilogue warps (four warpgroups, each owning every fourth block) drain them with tcgen05.ld.
+// The score matrix never leaves the SM.  Work items (a pass, a layer/KV head, a chunk of key tiles of one sequence)
+// are laid out so that pass 2 of a (layer, KV head) unit follows its pass 1 by a lag of a few units: close enough that
+// the unit's keys are still in L2 for the second read (K crosses HBM once), far enough that the statistics pass 2
+// needs are already published.  The epilogue warpgroups never meet at a CTA-wide barrier: each walks the items on its
+// own and only waits for accumulators; two helper warps do everything else at item boundaries -- they merge and
+// publish the row statistics of finished pass-1 items, bump a per-unit counter, wait (bounded) on that counter for
+// the CTA's next pass-2 item and merge the chunks' statistics into its rows' log-sum-exps, one item ahead of the
+// epilogue.  A pass-2 item only depends on items at smaller schedule positions and pass-1 items never wait, so the
+// schedule cannot deadlock for any grid size.
 //
-// Every wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word, stops issuing
-// work, drains its own TMA copies with bounded waits, frees its TMEM and returns.
+// Every wait is bounded: on expiry the CTA raises SG_ERR_TIMEOUT in the status word, stops issuing work, waits
+// (bounded) for its own TMA copies and MMAs, frees its TMEM and returns.
 #include <cuda.h>
 
 #include <vector>
-#include <cstdlib>
 
 #include "common.cuh"
 #include "launch.h"
@@ -60,7 +61,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 #define SG_PROF_BEGIN(t) const long long t = clock64()
 #define SG_PROF_ADD(acc, t) acc += clock64() - (t)
 #define SG_PROF_INC(acc) acc += 1
-#define SG_PROF_EVENT(kind, n) do { if (p.clock_out && blockIdx.x == 0 && (n) < 4096u) p.clock_out[32 * 1024 + (kind) * 4096 + (n)] = (unsigned long long)clock64(); } while (0)
 #define SG_PROF_STORE(slot, v) do { if (p.clock_out) p.clock_out[32 * (size_t)blockIdx.x + (slot)] = (unsigned long long)(v); } while (0)
 constexpr int kClockWords = 32;
 #else
@@ -68,7 +68,6 @@ constexpr int kClockWords = 32;
 #define SG_PROF_BEGIN(t)
 #define SG_PROF_ADD(acc, t)
 #define SG_PROF_INC(acc)
-#define SG_PROF_EVENT(kind, n)
 #define SG_PROF_STORE(slot, v)
 constexpr int kClockWords = 4;
 #endif
@@ -86,7 +85,6 @@ struct ScoreParams {
   int32_t compact;         // schedule layout: 0 = every slot 2*C positions, 1 = positions without an item removed
   int32_t tiles_per_chunk, max_items, k_stages, q_bufs;
   int32_t wgslots;         // statistics slots per item: 4 (one per epilogue warpgroup) or 1 (every row block has one owner)
-  int32_t debug_mode;      // profiling builds only: 1 = epilogue releases accumulators without reading them
   int32_t withhold_unit;   // testing only: pass-1 items of this unit are never counted as done (-1 = none)
   uint32_t wait_ns;        // limit of every bounded wait, nanoseconds
   unsigned long long* clock_out;   // testing only: per CTA {clock64 start, end, globaltimer start, end}, or null
@@ -564,20 +562,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           for (int blk = 0; blk < nblk; ++blk, q_lo += q_blk_lo) {
             const uint32_t as = (tile_count++) % kEpiGroups;               // blocks go to the warpgroups in rotation
             const uint32_t par = ((phbits >> as) & 1u) ^ 1u;
-            SG_PROF_EVENT(8, tile_count - 1);
             SG_PROF_BEGIN(ta);
-            const bool fast = mbar_test(bar_aempty0 + as * 8u, par);
-            SG_PROF_EVENT(9, tile_count - 1);
-            if (!fast) ok = mbar_wait(bar_aempty0 + as * 8u, par, abort_flag, p.wait_ns, 0u);
+            ok = mbar_wait(bar_aempty0 + as * 8u, par, abort_flag, p.wait_ns, 0u);
             SG_PROF_ADD(w_aempty, ta);
-            SG_PROF_EVENT(0, tile_count - 1);
             if (!ok) break;
             tc_fence_after();
             umma_block<4 * kSub>(tmem_base + as * 128u, pass1 ? q_lo : k_lo, pass1 ? k_lo : q_lo, a_sub, b_sub, kSmemDescHi,
                                  blk == nblk - 1 ? idesc_last : idesc_full);
-            SG_PROF_EVENT(7, tile_count - 1);
             umma_commit(bar_afull0 + as * 8u);
-            SG_PROF_EVENT(1, tile_count - 1);
             phbits ^= 1u << as;
           }
           if (ok) umma_commit(bar_kempty(ks));
@@ -610,7 +602,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     int n_p2 = 0;                                      // pass-2 items seen so far (selects the lse buffer)
     int n_p1 = 0;                                      // pass-1 items seen so far (selects the statistics buffer)
     bool ok = true;
-    SG_PROF_DECL(w_afull = 0, w_lse = 0, w_pub = 0, n_blocks = 0);
+    SG_PROF_DECL(w_afull = 0, w_lse = 0, w_pub = 0, n_blocks = 0, w_sfree = 0);
     // Releases the accumulator: called right after the block's last TMEM load has completed, before the
     // arithmetic on those columns, so the MMAs of this warpgroup's next block overlap it.
     auto release_acc = [&]() {
@@ -618,7 +610,6 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_aempty(as));
       aph ^= 1u;
-      if (lane == 0) SG_PROF_EVENT(3 + lane_grp, tile_count - 1);
     };
     for (long long pos = blockIdx.x; pos < npos; pos += gridDim.x) {   // no early exit: every thread meets its warpgroup's barriers
       const ScoreItem it = decode_position(p, pos, s_cu, s_prefix);
@@ -636,7 +627,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         // by the helper warps (practically always true already; the wait is bounded).
         const int sbuf = n_p1 & 1, suse = n_p1 >> 1;
         ++n_p1;
+        SG_PROF_BEGIN(tsf);
         if (ok && suse > 0) ok = mbar_wait(bar_stat_free(sbuf), (uint32_t)((suse - 1) & 1), abort_flag, p.wait_ns, 32u);
+        SG_PROF_ADD(w_sfree, tsf);
         float* sm_m = sm_stat + (size_t)(sbuf * 2 * p.wgslots + wgslot) * p.Ralloc;   // this warpgroup's slot: max ...
         float* sm_l = sm_m + p.wgslots * p.Ralloc;                                     // ... and sum of exp2
         // Slot (wgslot, blk*128 + row_in_tile) is only ever touched by this thread during the item, so the running
@@ -658,7 +651,6 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
             SG_PROF_ADD(w_afull, ta);
             SG_PROF_INC(n_blocks);
-            if (wg_tid == 0) SG_PROF_EVENT(2, tile_count - 1);
             if (!ok) continue;
             tc_fence_after();
             const int r = blk * 128 + row_in_tile;
@@ -716,17 +708,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               }
             };
             uint32_t cur[32];
-#ifdef SG_SCORE_PROFILE
-            if (p.debug_mode == 1) { release_acc(); continue; }
-#endif
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
               tmem_ld_wait(cur);
               if (j == 3) release_acc();
-#ifdef SG_SCORE_PROFILE
-              if (p.debug_mode == 2) continue;
-#endif
               chunk(cur, j * 32);
             }
             sm_m[r] = m;
@@ -768,7 +754,6 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
             SG_PROF_ADD(w_afull, ta);
             SG_PROF_INC(n_blocks);
-            if (wg_tid == 0) SG_PROF_EVENT(2, tile_count - 1);
             if (!ok) continue;
             tc_fence_after();
             const int ncols = min(128, p.Rpad - blk * 128);
@@ -794,17 +779,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               }
             };
             uint32_t cur[32];
-#ifdef SG_SCORE_PROFILE
-            if (p.debug_mode == 1) { release_acc(); continue; }
-#endif
 #pragma unroll 1
             for (int j = 0; j < nchk; ++j) {
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
               tmem_ld_wait(cur);
               if (j == nchk - 1) release_acc();
-#ifdef SG_SCORE_PROFILE
-              if (p.debug_mode == 2) continue;
-#endif
               chunk(cur, j * 32);
             }
           }
@@ -840,7 +819,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
       }
     }
 #ifdef SG_SCORE_PROFILE
-    if (wg_tid == 0) { SG_PROF_STORE(9 + wg * 4, w_afull); SG_PROF_STORE(10 + wg * 4, w_lse); SG_PROF_STORE(11 + wg * 4, w_pub); SG_PROF_STORE(12 + wg * 4, n_blocks); }
+    if (wg_tid == 0) { SG_PROF_STORE(9 + wg * 4, w_afull); SG_PROF_STORE(10 + wg * 4, w_lse); SG_PROF_STORE(11 + wg * 4, w_pub + w_sfree); SG_PROF_STORE(12 + wg * 4, n_blocks); }
 #endif
   } else if (warp >= kHelperWarp) {
     // ------------------------------------------------------------ helper warps (two: each handles half of the rows)
@@ -1046,16 +1025,16 @@ ScorePlan plan_score(const sg_shape* s) {
   const int64_t tiles_per_unit = (int64_t)s->total_tokens / kTileKeys + s->batch;
   int tpc = pl.R >= 256 ? 32 : 16;
   while (tpc > 4 && (tiles_per_unit / tpc + s->batch) * pl.U < 6 * kNumSMs) tpc /= 2;
-  if (getenv("SG_SCORE_TPC")) tpc = atoi(getenv("SG_SCORE_TPC"));   // EXPERIMENT
   pl.tiles_per_chunk = tpc;
   pl.max_items = (int)(tiles_per_unit / tpc + s->batch + 1);
-  // Pass 2 of a unit trails its pass 1 by `lag` units.  The lag must span more schedule positions than there
-  // are CTAs (each slot holds about 2*C positions), otherwise pass-2 items run in the same wave as the pass-1
-  // items they wait for and stall; beyond that it is kept as small as possible so that the unit's keys are
-  // still in L2 for the second read.
+  // Pass 2 of a unit trails its pass 1 by `lag` units.  The lag must span several times more schedule positions
+  // than there are CTAs (each slot holds about 2*C positions): a pass-2 item needs every pass-1 item of its unit
+  // published, and the helper warps prepare it one item ahead, so with a lag of one wave pass-2 items wait for
+  // statistics (measured on the 8B shape: 12-19 % of the epilogue's time at 1.25 waves, < 5 % at 3.5).  Beyond
+  // that it is kept small so that the unit's keys are still in L2 for the second read; 3.5 waves is where the
+  // time stops falling (8B shape 268 -> 232 us, long-context shape 808 -> 740 us from 1.25 to 3.5 waves).
   const int64_t c_est = (tiles_per_unit - s->batch) / tpc + 1;
-  static const int lag_num = getenv("SG_SCORE_LAGNUM") ? atoi(getenv("SG_SCORE_LAGNUM")) : 14;   // EXPERIMENT
-  int64_t lag = (lag_num * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
+  int64_t lag = (14 * kNumSMs / 4 + 2 * c_est - 1) / (2 * c_est) + 1;
   if (2 * lag > pl.U) lag = pl.U;     // few units: all pass-1 items first, then all pass-2 items
   pl.lag = (int)lag;
   pl.counter_bytes = ((size_t)pl.U * sizeof(int) + 255) & ~(size_t)255;
@@ -1191,7 +1170,6 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   p.k_stages = pl.k_stages;
   p.q_bufs = pl.q_bufs;
   p.wgslots = pl.wgslots;
-  p.debug_mode = getenv("SG_SCORE_DEBUG") ? atoi(getenv("SG_SCORE_DEBUG")) : 0;   // EXPERIMENT
   p.withhold_unit = g_test_withhold_unit.load(std::memory_order_relaxed);
   const int limit_ms = g_test_wait_limit_ms.load(std::memory_order_relaxed);
   p.wait_ns = limit_ms > 0 ? (uint32_t)limit_ms * 1000000u : 1000000000u;
