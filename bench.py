@@ -396,6 +396,130 @@ def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (
         torch.cuda.empty_cache()
     return out
 
+def _graph_us(fn, dev, reps=7):
+    """Median device time (us) of `fn` replayed from a CUDA graph on a side stream (CUDA events on that stream)."""
+    import torch
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        fn(); side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+        g.replay(); side.synchronize()
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side); g.replay(); e1.record(side); side.synchronize()
+            ts.append(e0.elapsed_time(e1))
+    return 1e3 * float(np.median(ts))
+
+
+def score_clock(dev, hp, d_q, d_k):
+    """SM clock (MHz) the scoring kernel really runs at: every CTA records clock64 and globaltimer at its start and end
+    (testing hook of the library); a 200 ms nvidia-smi sample cannot see a kernel of a fraction of a millisecond."""
+    import torch
+    from paper_2607_28150_b200 import binding as sg
+    grid = max(1, sg.sg_testing_score_grid(hp.shape))
+    buf = torch.zeros(32 * grid, dtype=torch.int64, device=dev)
+    for _ in range(2):
+        hp.score(d_q, d_k)                       # same thermal / power state as the timed calls
+    torch.cuda.synchronize()
+    try:
+        sg.sg_testing_score_clock(buf)
+        hp.score(d_q, d_k)
+        torch.cuda.synchronize()
+    finally:
+        sg.sg_testing_score_clock(None)
+    rec = buf.cpu().numpy()[: 4 * grid].reshape(grid, 4).astype(np.float64)
+    cyc, ns = rec[:, 1] - rec[:, 0], rec[:, 3] - rec[:, 2]
+    ok = (cyc > 0) & (ns > 0)
+    return float(1e3 * np.median(cyc[ok] / ns[ok])) if ok.any() else None
+
+
+def measure_config(dev, peaks, cfg, fractions=None, decode=True):
+    """Every stage of the path on one benchmark configuration, each timed alone (CUDA graph replay, CUDA events, median
+    of 7): sg_score, sg_select_topk, sg_pack_kv, sg_select_pack_kv over all the configuration's layers in one call each,
+    and one sg_sparse_decode_attn call (layer 0).  Inputs are the seeded synthetic caches of the workload recipe,
+    resident in HBM.  Returns per stage: time, algorithmic bytes / flops, achieved rate, the roof that binds, frac."""
+    import torch
+    from paper_2607_28150_b200 import binding as sg, workloads as wl
+    from paper_2607_28150_b200.pipeline import HotPath, as_device
+    L, B, Hq, Hkv, d, W = cfg.num_layers, cfg.batch, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.window
+    T = cfg.total_tokens
+    d_q = torch.empty((L, B, W, Hq, d), dtype=torch.int16, device=dev)
+    d_k = torch.empty((L, T, Hkv, d), dtype=torch.int16, device=dev)
+    d_v = torch.empty((L, T, Hkv, d), dtype=torch.int16, device=dev)
+    for l in range(L):
+        lay = wl.make_layer(cfg, l)
+        d_q[l] = as_device(lay["q_win"], dev); d_k[l] = as_device(lay["k"], dev); d_v[l] = as_device(lay["v"], dev)
+    tc_peak, hbm_peak = peaks["bf16_tflops_sustained"], peaks["hbm_gbs"]
+    out = {"workload": "%s: L=%d B=%d Hq=%d Hkv=%d d=%d W=%d T=%d" % (cfg.name, L, B, Hq, Hkv, d, W, T), "stages": {}}
+
+    def hbm(nbytes, us):
+        a = nbytes / us / 1e3
+        return {"us": us, "bytes": nbytes, "achieved": a, "unit": "GB/s", "bound": "hbm", "peak": hbm_peak, "frac": a / hbm_peak}
+
+    first = True
+    for frac in (fractions or [None]):
+        budgets = cfg.budgets(frac) if frac is not None else cfg.budgets()
+        hp = HotPath(L, Hq, Hkv, d, W, cfg.seqlens, budgets, device=dev)
+        nloc = cfg.n_local(frac) if frac is not None else cfg.n_local()
+        work = algorithmic_work(cfg if frac is None else wl.varlen(frac, L, cfg.seqlens), nloc)
+        tag = "" if frac is None else "@%g%%" % (100 * frac)
+        if first:
+            us = _graph_us(lambda: hp.score(d_q, d_k), dev)
+            r = hbm(work["score"]["bytes"], us)
+            tf = work["score"]["flops"] / us / 1e6
+            exps = 2.0 * work["score"]["flops"] / (2.0 * d)
+            mhz = score_clock(dev, hp, d_q, d_k)
+            r.update(tensor_tflops=tf, tensor_frac_of_sustained=tf / tc_peak, sfu_exp_per_s=exps / (us * 1e-6), sm_mhz_in_kernel=mhz,
+                     sfu_frac_at_kernel_clock=(exps / (us * 1e-6)) / (16.0 * 148 * mhz * 1e6) if mhz else None)
+            if cfg.group * W > tc_peak * 1e3 / hbm_peak:                  # above the ridge: tensor cores bind
+                r.update(bound="tensor", achieved=tf, unit="TFLOP/s", peak=tc_peak, frac=tf / tc_peak)
+            out["stages"]["score"] = r
+        else:
+            hp.score(d_q, d_k)
+        torch.cuda.synchronize()
+        out["stages"]["select" + tag] = hbm(work["select"]["bytes"], _graph_us(lambda: hp.select(), dev))
+        out["stages"]["pack" + tag] = hbm(work["pack"]["bytes"], _graph_us(lambda: hp.pack(d_k, d_v), dev))
+        out["stages"]["select_pack" + tag] = hbm(work["select"]["bytes"] + work["pack"]["bytes"],
+                                                  _graph_us(lambda: hp.select_pack(d_k, d_v), dev))
+        if decode and first:
+            sel_host = hp.sel_idx[0].cpu().numpy()
+            _, _, loc, cl = wl.make_index_split(cfg, 0, 0, budgets, nloc, exclude=sel_host, cu_excl=hp.cu_k_host)
+            NL = int(cl[-1])
+            qd = as_device(wl.make_decode_queries(cfg, 0, 0), dev)
+            d_loc, d_cl = (as_device(loc, dev) if NL else None), as_device(cl, dev)
+            o = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=dev)
+            hp.decode_workspace(NL)
+            calls = 8
+
+            def dec():
+                for _ in range(calls):
+                    hp.decode(0, qd, d_k[0], d_v[0], d_loc, d_cl, NL, o)
+            us = _graph_us(dec, dev) / calls
+            r = hbm(work["decode_call"]["bytes"], us)
+            r["note"] = "one call (layer 0), %d back-to-back calls per graph, same buffers: warm L2 below 126 MB" % calls
+            r["tokens_per_s"] = B / (us * 1e-6)
+            out["stages"]["decode_call"] = r
+        out["dev_status" + tag] = hp.read_status()
+        first = False
+        del hp
+    del d_q, d_k, d_v
+    torch.cuda.empty_cache()
+    return out
+
+
+def measure_configs(dev, peaks):
+    """c1 (tiny), c3 (ragged batch, one layer: budgets 10 % with every stage, 5 % and 20 % for selection and gather) and
+    c4 (long context, 8 layers) measured in the same run as the timed c2 step."""
+    from paper_2607_28150_b200 import workloads as wl
+    return {
+        "c1": measure_config(dev, peaks, wl.tiny()),
+        "c3": measure_config(dev, peaks, wl.varlen(0.10), fractions=[0.10, 0.05, 0.20]),
+        "c4": measure_config(dev, peaks, wl.llama70b()),
+    }
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -619,7 +743,7 @@ def run_ours(args):
     sp_bytes = work["select"]["bytes"] + work["pack"]["bytes"]
     value = world * sp_bytes / (st["select_pack"] * 1e-3) / 1e9
     dec_tok = world * B * nsteps_dec / (st["decode"] * 1e-3) if nsteps_dec else None
-    e2e_value = world * sp_bytes / ((st_e["h2d"] + st_e["select_pack"] + st_e["d2h"]) * 1e-3) / 1e9
+    e2e_value = world * sp_bytes / ((st_e["h2d"] + st_e["score"] + st_e["select_pack"] + st_e["d2h"]) * 1e-3) / 1e9
     e2e_dec_tok = world * B * nsteps_dec / (st_e["decode"] * 1e-3) if nsteps_dec else None
     h2d = (h_q.numel() + h_k.numel() + h_v.numel()) * 2 + (h_qdec.numel() * 2 + (h_idx.numel() * 4 if NL else 0))
     d2h = (h_pk.numel() + h_pv.numel()) * 2 + h_sel.numel() * 4 + h_out.numel() * 2
@@ -650,6 +774,9 @@ def run_ours(args):
     sfu_peak = 16.0 * 148 * 1.965e9
     roofs["score"]["sfu_exp_per_s"] = exps / (st["score"] * 1e-3)
     roofs["score"]["sfu_frac_at_max_clock"] = roofs["score"]["sfu_exp_per_s"] / sfu_peak
+    mhz = score_clock(dev, hp, d_q, d_k)
+    roofs["score"]["sm_mhz_in_kernel"] = mhz
+    roofs["score"]["sfu_frac_at_kernel_clock"] = roofs["score"]["sfu_exp_per_s"] / (16.0 * 148 * mhz * 1e6) if mhz else None
     R = cfg.group * W
     if R > peaks["bf16_tflops_sustained"] * 1e3 / peaks["hbm_gbs"]:       # above the ridge: tensor cores bind
         roofs["score"].update(bound="tensor", achieved=roofs["score"]["tensor_tflops"], peak=tc_peak, unit="TFLOP/s",
@@ -677,11 +804,12 @@ def run_ours(args):
     next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 and not args.no_extras else None
     layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
     first_two = full_first_two_timing(dev, cfg, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
-    sweep = None
+    sweep, configs = None, None
     if args.workload == "c2" and not args.no_decode_sweep and not args.no_extras and world == 1:
         del d_k, d_v, h_k, h_v
         torch.cuda.empty_cache()
         sweep = decode_sweep_points(dev, peaks)
+        configs = measure_configs(dev, peaks)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
@@ -698,7 +826,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (2 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "decode_sweep": sweep, "next_rows": next_rows, "prefill_layerwise": layerwise, "prefill_full_first_two": first_two,
+        "decode_sweep": sweep, "configs": configs, "next_rows": next_rows, "prefill_layerwise": layerwise, "prefill_full_first_two": first_two,
         "e2e_pipelined": None if ms_pipe is None else {
             "ms_prefill": ms_pipe, "value": sp_bytes / (ms_pipe * 1e-3) / 1e9, "unit": UNIT,
             "note": "host buffers, layer by layer on three streams (copy in | score, select, pack | copy out); "
@@ -748,8 +876,26 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # Started as a plain process (not under torchrun): start the N replicas here, one process per GPU.  They
+        # exchange nothing but a barrier and the maximum of their device times; rank 0 prints the line.
+        import torch
+        from paper_2607_28150_b200 import replicas
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            raise SystemExit("bench.py --gpus %d: only %d CUDA device(s) visible" % (args.gpus, have))
+        env = dict(os.environ)
+        env.setdefault("NCCL_DEBUG", "INFO")             # the communicator's one log line (ring/tree, NVLS) goes to stderr
+        env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+        codes, out0 = replicas.launch_local_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env)
+        sys.stdout.write(out0)
+        sys.stdout.flush()
+        if any(codes):
+            raise SystemExit("bench.py: rank exit codes %s" % codes)
+        return
+    run_ours(args)
 
 
 if __name__ == "__main__":

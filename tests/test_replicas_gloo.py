@@ -44,3 +44,34 @@ def test_single_process_is_identity():
     from paper_2607_28150_b200 import replicas
     assert replicas.max_over_ranks({"a": 3.0}) == {"a": 3.0}
     assert replicas.aggregate_throughput(10.0, 2.0) == 5.0
+
+
+_RANK_PROGRAM = r'''
+import json, os, sys
+sys.path.insert(0, sys.argv[1])
+import torch.distributed as dist
+from paper_2607_28150_b200 import replicas
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]) == rank
+dist.init_process_group("gloo")
+mx = replicas.max_over_ranks({"step": 5.0 + rank})
+dist.barrier()
+if rank == 0:
+    print(json.dumps({"n_gpus": replicas.world(), "ms": mx["step"], "value": replicas.aggregate_throughput(10.0, mx["step"])}))
+dist.destroy_process_group()
+'''
+
+
+def test_launcher_starts_one_rank_per_replica_and_returns_rank_zero_output(tmp_path):
+    """`bench.py --gpus N` started as a plain process spawns its N ranks with this launcher; here the ranks are CPU
+    processes on gloo: both must start, rendezvous on 127.0.0.1, and rank 0's single line must carry world size 2."""
+    import json
+    import sys
+    from paper_2607_28150_b200 import replicas
+    prog = tmp_path / "rank.py"
+    prog.write_text(_RANK_PROGRAM)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    codes, out = replicas.launch_local_ranks(2, [sys.executable, str(prog), root], timeout=180)
+    assert codes == [0, 0]
+    line = json.loads(out.strip().splitlines()[-1])
+    assert line == {"n_gpus": 2, "ms": 6.0, "value": 2 * 10.0 / 6.0}
