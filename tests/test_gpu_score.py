@@ -97,3 +97,26 @@ def test_score_strided_cache():
     ws = sg.alloc_workspace(sg.SG_OP_SCORE, shp)
     sg.sg_score(shp, gpu_ops.dev(q), gpu_ops.dev(kbig), imp, ws)
     assert_close(imp.cpu().numpy(), oracle.score(q, k, cu))
+
+
+def test_score_late_key_far_above_everything_before_it():
+    """A key whose score lies more than 2^127 (in exp2 terms) above every earlier key of its row, met in the SECOND
+    key tile a warpgroup sees within a work item: pass 1 sums each chunk against a running reference that is only
+    refreshed when the sum leaves the safe range, so this is the case where it must be refreshed (the unguarded sum
+    would be +inf).  The shape has enough (layer, head) units that work items span eight key tiles, two per
+    warpgroup.  Also the mirror case, a dominant key first and tiny ones after it."""
+    import gpu_ops
+    from paper_2607_28150_b200.workloads import f32_to_bf16_bits
+    rng = np.random.default_rng(9)
+    L, N, W, Hq, Hkv, d = 32, 4096, 8, 8, 8, 64
+    cu = cu_of((N,))
+    for where in (5 * 128 + 20, 3):
+        qv = rng.standard_normal((L, Hkv, d)).astype(np.float32)
+        q = np.broadcast_to(qv[:, None, None], (L, 1, W, Hq, d)).copy()
+        k = (0.01 * rng.standard_normal((L, N, Hkv, d))).astype(np.float32)
+        k[:, where] = 20.0 * qv                     # score ~ 20 |q|^2 / sqrt(d) ~ 160 nats above the rest
+        qb, kb = f32_to_bf16_bits(q), f32_to_bf16_bits(k)
+        want = oracle.score(qb, kb, cu)
+        got = gpu_ops.score(qb, kb, cu)
+        assert_close(got, want)
+        assert np.all(np.isfinite(got)) and np.abs(got[:, :, where] - W).max() < 1e-2
