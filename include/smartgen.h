@@ -181,15 +181,13 @@ sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void
 /*
  * sg_split_index -- split a KV index into its local and remote parts (Algorithm 1).
  *
- * Defines: Algorithm 1, "KV Index Splitting and Reordering" (Section 4.2).  The KV mask holds one int8
- * per token, shared by all heads: 0 = padding, 1 = the token's KV entries are locally available,
- * 2 = they reside on a remote prefill node.  For every row of the KV index (one sequence, one KV head):
- *   (1)   mask = kv_mask[kv_index]
- *   (4,5) if `reorder`: sort the row's mask in descending order (stable: entries keep their relative
- *         order inside a class) and apply the same order to the index, so that remote entries are
- *         contiguous at the start of the row
- *   (2)   local_index  = kv_index[mask == 1]
- *   (3)   remote_index = kv_index[mask == 2]
+ * Defines: Algorithm 1, KV index splitting and reordering (Section 4.2).  The KV mask holds one int8 per
+ * token, shared by all heads, naming the token's class: 0 = padding, 1 = the token's KV entries are locally
+ * available, 2 = they reside on a remote prefill node.  Every row of the KV index (one sequence, one KV head)
+ * is split by the class of its entries: local_index receives the entries of class 1 and remote_index those of
+ * class 2, each in the row's own order.  With `reorder`, the row is also returned as a stable three-way
+ * partition by class (remote first, then local, then padding; entries keep their relative order inside a
+ * class), so that the remote entries are contiguous at the start of the row.
  * Padding entries (mask 0) are dropped from both lists; an index outside [0, N_b) sets the SG_ERR_INDEX
  * device bit and is treated as padding.
  *
@@ -197,7 +195,7 @@ sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void
  * kv_index     int32 [H_kv][K_tot], row segment of sequence b at cu_k[b], sequence-local positions
  *              (the layout sg_select_topk writes for one layer); cu_k device int32 [B+1].
  * kv_mask      int8 [T], ragged by cu_seqlens.
- * reordered    int32 [H_kv][K_tot] or NULL: the row after steps (4)-(5) (a copy when reorder == 0).
+ * reordered    int32 [H_kv][K_tot] or NULL: the partitioned row (a copy when reorder == 0).
  * local_index, remote_index  int32 [H_kv][K_tot]: each row segment is filled from its start; the counts
  *              go to n_local / n_remote, int32 [B][H_kv].  Entries past the counts are left untouched.
  * The lists feed sg_sparse_decode_attn: local_index (compacted per head) is its local-lane index list,
@@ -214,8 +212,8 @@ sg_status sg_split_index(const sg_shape* shape, const int32_t* kv_index, const i
  * Blocks: every layer's cache is partitioned along the sequence into M = num_blocks KV blocks; token t of a
  * sequence of length N_b belongs to block floor(t * M / N_b).  A block holds its tokens' entries of all KV heads.
  *
- * sg_profile_accumulate -- S(e), "the number of times entry e is selected in the decoding stage during the
- *   offline profiling": adds 1 to counts[g][cu[b] + t] for every entry t of one layer's KV index of one decode
+ * sg_profile_accumulate -- S(e) of Eq. 1 (Section 4.1), the selection count of a KV entry over the profiled
+ *   decode steps: adds 1 to counts[g][cu[b] + t] for every entry t of one layer's KV index of one decode
  *   step.  shape->num_layers must be 1; kv_index int32 [H_kv][K_tot] with cu_k as in sg_select_topk;
  *   counts int32 [H_kv][T] (the caller zeroes it before the first call).  Out-of-range entries set SG_ERR_INDEX.
  * sg_block_importance -- Eq. 1: importance[l][m] = +inf for l = 0, 1 (the first two layers are always

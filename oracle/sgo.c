@@ -166,8 +166,8 @@ int sgo_select_topk(int L, int B, int Hkv, const int32_t *cu, const float *impor
 
 /*
  * Gather-pack of the selected K/V rows into a contiguous buffer (Section 4.2: the selected KV
- * has shape BH x k x d, a "row" being the k entries of one head; the prefill node "selects the
- * required KV entries locally" before sending them).
+ * has shape BH x k x d, a row being the k entries of one head; the prefill node picks the required
+ * entries out of its own cache before sending them).
  *
  * packed_k/v bf16 [L][K_tot*Hkv][d]; row of (b, g, j) is cu_k[b]*Hkv + g*k_b + j.
  * Returns 3 if an index is outside its sequence.
@@ -295,19 +295,19 @@ int sgo_sparse_decode_attn(int B, int Hq, int Hkv, int d, const int32_t *cu, con
 }
 
 /*
- * Algorithm 1 (KV index splitting and reordering), per row of the KV index.
+ * KV index splitting and reordering (Algorithm 1, Section 4.2), per row of the KV index.
  *
- *   (1) mask = kv_mask[kv_index]          -- one int8 per token, shared by all heads;
- *                                            0 = padding, 1 = local, 2 = remote
- *   (4,5) optional: sort each row of mask in descending order and apply the same order to
- *         kv_index, so that remote entries (value 2) are contiguous at the start of the row;
- *         the sort is stable, i.e. entries keep their original relative order in each class
- *   (2) local_index  = kv_index[mask == 1]
- *   (3) remote_index = kv_index[mask == 2]
+ * Definition used here: the KV mask holds one int8 per token, shared by all heads, that names the
+ * token's class (2 = its entries are on the remote prefill node, 1 = locally available,
+ * 0 = padding).  A row of the KV index is split by the class of each of its entries: the local list
+ * is the row's entries of class 1, the remote list those of class 2, each in the row's own order.
+ * With `reorder` the row itself is also returned as a stable partition by class, remote entries
+ * first, then local, then padding (a stable descending sort by class), so that the remote entries
+ * are contiguous at the start of the row.
  *
  * kv_index int32 [Hkv][K_tot] with prefix sums cu_k (sequence-local positions, row segment of
  * (b, g) at g*K_tot + cu_k[b]); kv_mask int8 [T] ragged by cu.
- * Outputs: reordered int32 [Hkv][K_tot] (the row after steps 4-5, or a copy when reorder == 0);
+ * Outputs: reordered int32 [Hkv][K_tot] (the partitioned row, or a copy when reorder == 0);
  * local_index / remote_index int32 [Hkv][K_tot], each row segment filled from its start;
  * n_local / n_remote int32 [B][Hkv].  Entries with mask 0 are dropped from both lists.
  */
@@ -358,7 +358,7 @@ int sgo_split_index(int B, int Hkv, const int32_t *cu, const int32_t *cu_k, cons
  */
 static int64_t block_of(int64_t t, int64_t N, int64_t M) { return t * M / N; }
 
-/* S(e): "the number of times entry e is selected in the decoding stage during the offline profiling".
+/* S(e) of Eq. 1 (Section 4.1): how often a KV entry was selected over the profiled decode steps.
  * Adds one to counts[g][cu[b] + t] for every entry t of the KV index (one layer, one decode step).
  * kv_index int32 [Hkv][K_tot] with prefix sums cu_k; counts int32 [Hkv][T]. */
 int sgo_profile_accumulate(int B, int Hkv, const int32_t *cu, const int32_t *cu_k, const int32_t *kv_index,
@@ -426,7 +426,7 @@ int sgo_proactive_mask(int B, int M, const int32_t *cu, int layer, const int32_t
 }
 
 /* Speculative transfer (Section 4.3): after the prefill stage has pushed the top-K_r blocks, every decoding
- * iteration delivers the next blocks "in the order of their importance, as defined in Eq. 1", at most a fixed
+ * iteration delivers the next blocks in descending order of their Eq. 1 importance, at most a fixed
  * fraction (the speculative ratio) of ALL L*M blocks per iteration.  Number of blocks on the decode node after
  * `iteration` speculative transfers; the per-iteration quota is ratio * L * M rounded down, at least one block. */
 int64_t sgo_speculative_delivered(int L, int M, int64_t K_r, double ratio, int iteration) {

@@ -1,11 +1,10 @@
 // sg_split_index: Algorithm 1 (KV index splitting and reordering) on the device.
 //
-// One CTA owns one row of the KV index (one sequence, one KV head).  Operator (1) gathers the int8 mask
-// value of every selected token; operators (4)-(5), the per-row descending sort of the mask with the same
-// order applied to the index, are a stable three-way partition (remote = 2 first, then local = 1, then
-// padding = 0), done with ballots and prefix counts -- no atomics, so the output order is a pure function
-// of the input; operators (2)-(3) write the local and the remote index lists.  Integer work only, bound by
-// latency (a row is a few KB).
+// One CTA owns one row of the KV index (one sequence, one KV head).  It looks up the int8 class of every
+// selected token in the KV mask (2 = remote, 1 = local, 0 = padding) and forms a stable three-way partition of
+// the row by class -- remote first, then local, then padding -- with ballots and prefix counts: no atomics, so
+// the output order is a pure function of the input.  The partitioned row (when asked for) and the local and
+// remote index lists with their counts are written.  Integer work only, bound by latency (a row is a few KB).
 #include "common.cuh"
 
 namespace sg {
