@@ -414,6 +414,22 @@ def _graph_us(fn, dev, reps=7):
     return 1e3 * float(np.median(ts))
 
 
+def handover_timing(dev, hp, d_q, d_k, d_v):
+    """What the kernel boundary between scoring and selection costs: device time of sg_score and sg_select_pack_kv each
+    replayed alone, and of the two back to back in one graph.  `gap_us` = both - (score + select_pack) is everything a
+    score -> select fusion could remove (launch hand-over, drained SMs, and the importance array's trip through L2/HBM:
+    `importance_bytes` written once and read once)."""
+    a = _graph_us(lambda: hp.score(d_q, d_k), dev)
+    b = _graph_us(lambda: hp.select_pack(d_k, d_v), dev)
+
+    def both():
+        hp.score(d_q, d_k)
+        hp.select_pack(d_k, d_v)
+    c = _graph_us(both, dev)
+    imp_bytes = hp.importance.numel() * 4
+    return {"score_us": a, "select_pack_us": b, "back_to_back_us": c, "gap_us": c - a - b, "gap_frac_of_prefill": (c - a - b) / c,
+            "importance_bytes": imp_bytes, "importance_round_trip_us_at_copy_peak": 2 * imp_bytes / load_peaks()["hbm_gbs"] / 1e3}
+
 def score_clock(dev, hp, d_q, d_k):
     """SM clock (MHz) the scoring kernel really runs at: every CTA records clock64 and globaltimer at its start and end
     (testing hook of the library); a 200 ms nvidia-smi sample cannot see a kernel of a fraction of a millisecond."""
@@ -502,6 +518,8 @@ def measure_config(dev, peaks, cfg, fractions=None, decode=True):
             r["note"] = "one call (layer 0), %d back-to-back calls per graph, same buffers: warm L2 below 126 MB" % calls
             r["tokens_per_s"] = B / (us * 1e-6)
             out["stages"]["decode_call"] = r
+        if first:
+            out["score_select_handover"] = handover_timing(dev, hp, d_q, d_k, d_v)
         out["dev_status" + tag] = hp.read_status()
         first = False
         del hp
@@ -804,6 +822,7 @@ def run_ours(args):
     next_rows = next_rows_timing(dev, cfg, hp, d_k, d_v) if world == 1 and not args.no_extras else None
     layerwise = layerwise_prefill_timing(dev, hp, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
     first_two = full_first_two_timing(dev, cfg, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
+    handover = handover_timing(dev, hp, d_q, d_k, d_v) if world == 1 and not args.no_extras else None
     sweep, configs = None, None
     if args.workload == "c2" and not args.no_decode_sweep and not args.no_extras and world == 1:
         del d_k, d_v, h_k, h_v
@@ -826,7 +845,7 @@ def run_ours(args):
                 "ms_per_step": ms_e2e, "decode_tokens_per_s": e2e_dec_tok, "stage_ms": st_e, "steps": e2e_steps},
         "gpu_launches": args.steps * (2 + ncalls_dec),
         "roofline": dominant, "rooflines": roofs, "cpu_baseline": cpu, "clocks": clocks,
-        "decode_sweep": sweep, "configs": configs, "next_rows": next_rows, "prefill_layerwise": layerwise, "prefill_full_first_two": first_two,
+        "decode_sweep": sweep, "configs": configs, "next_rows": next_rows, "prefill_layerwise": layerwise, "prefill_full_first_two": first_two, "score_select_handover": handover,
         "e2e_pipelined": None if ms_pipe is None else {
             "ms_prefill": ms_pipe, "value": sp_bytes / (ms_pipe * 1e-3) / 1e9, "unit": UNIT,
             "note": "host buffers, layer by layer on three streams (copy in | score, select, pack | copy out); "

@@ -75,7 +75,7 @@ constexpr int kClockWords = 4;
 struct ScoreParams {
   const int32_t* cu;
   float* importance;
-  int* p1_done;            // [U] pass-1 items finished per unit (zeroed by the host call)
+  int* p1_done;            // [U] per unit: two counts per published pass-1 item, one per helper warp (zeroed by the host call)
   float2* part;            // [U][max_items][Ralloc] per-item row statistics (log2-domain max, sum of exp2)
   int32_t* dev_status;
   int64_t T;
@@ -373,8 +373,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   float* sm_part = sm_stat + 4 * p.wgslots * p.Ralloc;                // pass 2, several blocks per tile: [slots][groups][128] partial column sums
   const int part_slots = p.Rpad > 384 ? 4 : (p.Rpad > 128 ? 8 : 0);   // tiles in flight (see the pass-2 combine)
   int* sm_cnt = reinterpret_cast<int*>(sm_part + part_slots * kEpiGroups * 128);   // [kPartSlots][4 lane quarters] partials written
-  int* sm_icnt = sm_cnt + kPartSlots * 4;                             // [2] helper warps that stored their rows of the buffer's item (+ 6 spare words)
-  int* s_cu = sm_icnt + 8;                                            // [B+1]
+  int* s_cu = sm_cnt + kPartSlots * 4 + 8;                            // [B+1] (eight spare words before it)                                            // [B+1]
   int* s_prefix = s_cu + p.B + 1;                                     // [B+1]
 
   auto bar_qfull = [&](int s) { return smem_u32(&bars[s]); };
@@ -399,10 +398,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     for (int s = 0; s < kAccStages; ++s) { mbar_init(bar_afull(s), 1); mbar_init(bar_aempty(s), 4); }
     for (int s = 0; s < 2; ++s) { mbar_init(bar_lse_ready(s), 2); mbar_init(bar_lse_free(s), kEpiThreads / 32); }
     mbar_init(bar_drain, 1);
-    for (int s = 0; s < 2; ++s) { mbar_init(bar_stat_full(s), kEpiThreads / 32); mbar_init(bar_stat_free(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_stat_full(s), kEpiThreads / 32); mbar_init(bar_stat_free(s), 2); }
     *abort_flag = 0;
     for (int i = 0; i < kPartSlots * 4; ++i) sm_cnt[i] = 0;
-    for (int i = 0; i < 8; ++i) sm_icnt[i] = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
@@ -864,13 +862,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           for (int w = 0; w < p.wgslots; ++w) L += bl[w * p.Ralloc + r] * exp2f(bm[w * p.Ralloc + r] - Mu);
           p.part[slot + r] = make_float2(M, L);
         }
-        __threadfence();                               // this warp's stores, GPU-wide, before it reports in
+        // each helper warp counts its half of the rows itself (a unit is complete at 2*C counts): its stores are ordered
+        // before its count by the warp barrier plus one cumulative fence, and no hand-shake between the two warps is needed
         __syncwarp();
-        int second = 0;
-        if (lane == 0) second = atomicAdd(&sm_icnt[sbuf], 1);
-        second = __shfl_sync(0xffffffffu, second, 0);
-        if (second == 1 && lane == 0) {                  // both helper warps have stored their rows
-          sm_icnt[sbuf] = 0;
+        if (lane == 0) {
           __threadfence();
           if (!*abort_flag && it1.unit != p.withhold_unit) atomicAdd(p.p1_done + it1.unit, 1);
           mbar_arrive(bar_stat_free(sbuf));
@@ -887,7 +882,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           int cnt = 0;
           if (lane == 0) cnt = ld_acquire_gpu(p.p1_done + it2.unit);
           cnt = __shfl_sync(0xffffffffu, cnt, 0);
-          can = cnt >= C;
+          can = cnt >= 2 * C;
         }
         if (can) {
           SG_PROF_BEGIN(th2);
@@ -937,9 +932,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         }
       }
       if (progressed) { idle_since = 0; idle_iters = 0; continue; }
-      // nothing could run: sleep a little; every 16th idle round look at the abort flag and the clock (bounded wait)
-      __nanosleep(200);
-      if ((++idle_iters & 15u) == 0u) {
+      // nothing could run: sleep a little; every 64th idle round look at the abort flag and the clock (bounded wait)
+      __nanosleep(40);
+      if ((++idle_iters & 63u) == 0u) {
         if (*abort_flag) break;
         const uint64_t now = global_timer_ns();
         if (idle_since == 0) idle_since = now;
@@ -952,6 +947,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   }
 
   // ---------------------------------------------------------------- teardown
+  // This CTA has no work left: a kernel queued behind this one with programmatic stream serialization (the selection)
+  // may have its CTAs placed from now on; it still waits for this whole grid's completion before it reads anything.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   if (warp == kMmaWarp) {

@@ -43,8 +43,15 @@ __device__ __forceinline__ uint32_t order_key(uint32_t u) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// The selection kernels are launched with programmatic stream serialization: when the kernel before them in the
+// stream (normally the scoring kernel) lets its dependents go early, their CTAs are placed while it drains, and
+// the launch latency disappears behind it.  Nothing is read before this wait, which returns once that kernel has
+// completed and its writes are visible; after a kernel that does not take part it returns at once.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <bool kInSmem>
 __global__ void __launch_bounds__(kSelThreads, 1) select_topk_kernel(const SelParams p) {
+  pdl_wait();
   extern __shared__ __align__(16) uint32_t smem[];
   uint32_t* hist = smem;                              // [kHistCopies][256]
   uint32_t* total = hist + kHistCopies * 256;         // [256]
@@ -215,6 +222,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
 
 template <int E, int T, int PD>
 __global__ void __launch_bounds__(T) select_topk_reg_kernel(const SelParams p) {
+  pdl_wait();
   extern __shared__ __align__(16) uint32_t smem[];
   uint32_t* hist = smem;                               // [kRegCopies][kRegBins]
   uint32_t* wsum = hist + kRegCopies * kRegBins;       // [2][T/32]
@@ -462,13 +470,22 @@ namespace {
 sg_status select_launch(const sg_shape* shape, SelParams& p, bool fuse, void* stream) {
   const int64_t rows = (int64_t)shape->num_layers * shape->batch * shape->num_kv_heads;
   if (rows > 0x7fffffffLL) return SG_ERR_UNSUPPORTED;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)rows);
   const int pd = fuse ? shape->head_dim : 0;
 #define SG_LAUNCH_SELECT_REG_PD(E, T, PD)                                                       \
   do {                                                                                          \
     p.capacity = (E) * (T);                                                                     \
     SG_ENSURE_SMEM((select_topk_reg_kernel<E, T, PD>), (select_reg_smem_bytes<E, T>()));         \
-    select_topk_reg_kernel<E, T, PD><<<(unsigned)rows, T, select_reg_smem_bytes<E, T>(), s>>>(p); \
+    cfg.blockDim = dim3(T);                                                                     \
+    cfg.dynamicSmemBytes = select_reg_smem_bytes<E, T>();                                       \
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_topk_reg_kernel<E, T, PD>, p));                  \
   } while (0)
 #define SG_LAUNCH_SELECT_REG(E, T)                        \
   do {                                                    \
@@ -493,10 +510,14 @@ sg_status select_launch(const sg_shape* shape, SelParams& p, bool fuse, void* st
     const int smem = kSelFixedSmem + shape->max_seqlen * 4;
     p.capacity = shape->max_seqlen;
     SG_ENSURE_SMEM(select_topk_kernel<true>, smem);
-    select_topk_kernel<true><<<(unsigned)rows, kSelThreads, smem, s>>>(p);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = smem;
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_topk_kernel<true>, p));
   } else {
     p.capacity = 0;                                    // keys are re-read from global memory: any length
-    select_topk_kernel<false><<<(unsigned)rows, kSelThreads, kSelFixedSmem, s>>>(p);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = kSelFixedSmem;
+    SG_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_topk_kernel<false>, p));
   }
 #undef SG_LAUNCH_SELECT_REG
 #undef SG_LAUNCH_SELECT_REG_PD
