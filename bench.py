@@ -373,22 +373,29 @@ def decode_sweep_points(dev, peaks, points=((64, 0.20, 0.25), (128, 1.0, 0.0), (
                                                 d_loc, d_cl, NL, o)
         call()
         torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for _ in range(calls):
-                call()
-        g.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        best = float("inf")
-        for _ in range(3):
-            e0.record(); g.replay(); e1.record()
+        def graph_us_per_call():
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for _ in range(calls):
+                    call()
+            g.replay()
             torch.cuda.synchronize()
-            best = min(best, e0.elapsed_time(e1))
-        us = best * 1e3 / calls
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            best = float("inf")
+            for _ in range(3):
+                e0.record(); g.replay(); e1.record()
+                torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            return best * 1e3 / calls
+        us = graph_us_per_call()
+        try:
+            sg.sg_testing_decode_overlap(False)          # every call fully ordered behind the one before it
+            us_serial = graph_us_per_call()
+        finally:
+            sg.sg_testing_decode_overlap(True)
         nbytes = Hkv * (2 * (Ktot + NL) * d * 2 + NL * 4) + 2 * B * Hq * d * 2
         gbs = nbytes / us / 1e3
-        out.append({"batch": B, "sel": sel, "rho": rho, "n_sel": Ktot // B, "n_loc": NL // B, "us_per_call": us,
+        out.append({"batch": B, "sel": sel, "rho": rho, "n_sel": Ktot // B, "n_loc": NL // B, "us_per_call": us, "us_per_call_serialized": us_serial,
                     "bytes_per_call": nbytes, "l2": "larger than L2" if nbytes > 126e6 else "warm L2 (same buffers every call)",
                     "achieved_gbs": gbs, "frac_of_copy_peak": gbs / peaks["hbm_gbs"],
                     "tokens_per_s": B / (us * 1e-6)})
@@ -802,6 +809,21 @@ def run_ours(args):
     if ncalls_dec:
         roofs["decode"] = hbm("decode", work["decode_call"]["bytes"] * ncalls_dec, st["decode"], ncalls_dec)
         roofs["decode"]["us_per_call"] = 1e3 * st["decode"] / ncalls_dec
+        # the same calls, each fully ordered behind the one before it (no overlap of consecutive calls): what a model
+        # sees when the next layer's query depends on this layer's output
+        try:
+            sg.sg_testing_decode_overlap(False)
+            g_ser = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_ser):
+                decode_all(False)
+            g_ser.replay(); torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); g_ser.replay(); e1.record(stream); torch.cuda.synchronize()
+            roofs["decode"]["us_per_call_serialized"] = 1e3 * e0.elapsed_time(e1) / ncalls_dec
+        finally:
+            sg.sg_testing_decode_overlap(True)
+        roofs["decode"]["note"] = ("consecutive calls are independent (queries of all layers are inputs of the step) and overlap "
+                                   "up to their output stores; us_per_call_serialized: each call ordered behind the previous one")
     dominant = max(roofs.values(), key=lambda r: r["ms_per_step"])
 
     # ---- the oracle on the host cores, bounded sample

@@ -163,13 +163,15 @@ sg_status sg_select_pack_kv(const sg_shape* shape, const float* importance, cons
  *             scores.  A head with an empty list gets out = 0 and lse = -inf.
  * workspace   unused (split-KV partials are merged on chip); sg_workspace_bytes returns 0.
  *
- * Stream ordering: the kernel is launched with programmatic dependent launch and lets the next
- * kernel in the stream start early.  q is read, and out / lse are written, only after all earlier
- * work in the stream has completed.  The KV sources (packed_k/v, local_k/v), local_idx and the
- * prefix arrays (cu_seqlens, cu_k, cu_nloc) are treated as stable inputs of a decode step and may
- * be prefetched while an immediately preceding kernel THAT ITSELF OPTED IN to programmatic
- * dependent launch (such as the previous layer's sg_sparse_decode_attn) is still running: they
- * must not be outputs of such a kernel.  Ordinary preceding kernels are fully ordered as usual.
+ * Stream ordering: the kernel is launched with programmatic dependent launch and lets the next kernel
+ * in the stream start early.  out / lse are written only after all earlier work in the stream has completed.
+ * Every INPUT -- q, the KV sources (packed_k/v, local_k/v), local_idx, the per-head count arrays and the
+ * prefix arrays (cu_seqlens, cu_k, cu_nloc) -- is treated as a stable input of the decode step and may be
+ * read while an immediately preceding kernel THAT ITSELF OPTED IN to programmatic dependent launch (such as
+ * the previous layer's sg_sparse_decode_attn, or sg_score) is still running: inputs must not be outputs of
+ * such a kernel.  Ordinary preceding kernels (the projection that produces q, a copy, anything launched the
+ * usual way) are fully ordered before this call as usual.  Independent calls issued back to back therefore
+ * overlap everything but their output stores.
  */
 sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void* packed_k,
                                 const void* packed_v, const int32_t* cu_k, int32_t total_sel,

@@ -4,7 +4,7 @@
  * that tests can make a bounded device-side wait run out without hanging or faulting anything, and so
  * that the benchmark can read the SM clock a scoring kernel actually ran at.  The paper has no counterpart.
  *
- * All three are process-wide switches read by the next sg_score / sg_score_static call on any thread.
+ * All are process-wide switches read by the next call of the named entry point on any thread.
  */
 #ifndef SMARTGEN_TESTING_H_
 #define SMARTGEN_TESTING_H_
@@ -40,6 +40,14 @@ void sg_testing_score_clock(void* dev_buffer);
 
 /* Number of CTAs sg_score launches for this shape on a 148-SM device (the persistent grid). */
 int32_t sg_testing_score_grid(const sg_shape* shape);
+
+/*
+ * sg_testing_decode_overlap -- allowed = 0: the following sg_sparse_decode_attn calls are launched without
+ * programmatic stream serialization, i.e. fully ordered behind everything earlier in the stream, so that the
+ * benchmark can report the time of a call that may not overlap its predecessor; 1 (the default) restores the
+ * documented behaviour (a call overlaps the previous call up to its own output stores).
+ */
+void sg_testing_decode_overlap(int32_t allowed);
 
 #ifdef __cplusplus
 }

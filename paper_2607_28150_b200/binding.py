@@ -23,7 +23,7 @@ SG_OP_SCORE, SG_OP_SELECT_TOPK, SG_OP_PACK_KV, SG_OP_SPARSE_DECODE_ATTN, SG_OP_S
 EXPORTED = ("sg_workspace_bytes", "sg_score", "sg_select_topk", "sg_pack_kv", "sg_sparse_decode_attn",
             "sg_score_static", "sg_select_pack_kv", "sg_select_threshold", "sg_pack_kv_counted", "sg_sparse_decode_attn_counted", "sg_split_index", "sg_profile_accumulate", "sg_block_importance",
             "sg_transfer_budget", "sg_proactive_mask", "sg_push_blocks", "sg_speculative_delivered", "sg_strerror", "sg_last_cuda_error",
-            "sg_testing_score_fault", "sg_testing_score_clock", "sg_testing_score_grid")
+            "sg_testing_score_fault", "sg_testing_score_clock", "sg_testing_score_grid", "sg_testing_decode_overlap")
 SG_SCORE_STATIC_SCRATCH_BYTES = 8 << 20
 
 if not os.path.exists(LIB_PATH):
@@ -96,6 +96,8 @@ _lib.sg_testing_score_fault.restype = None
 _lib.sg_testing_score_fault.argtypes = [_i32, _i32]
 _lib.sg_testing_score_clock.restype = None
 _lib.sg_testing_score_clock.argtypes = [_vp]
+_lib.sg_testing_decode_overlap.restype = None
+_lib.sg_testing_decode_overlap.argtypes = [_i32]
 _lib.sg_testing_score_grid.restype = _i32
 _lib.sg_testing_score_grid.argtypes = [_sp]
 
@@ -109,6 +111,11 @@ def sg_testing_score_clock(buffer: Optional[torch.Tensor]) -> None:
     """Measurement hook: the next scoring kernels record their start/end clock64 and globaltimer per CTA into
     `buffer` (int64, at least 32 words per CTA); None switches it off."""
     _lib.sg_testing_score_clock(None if buffer is None else buffer.data_ptr())
+
+
+def sg_testing_decode_overlap(allowed: bool) -> None:
+    """Measurement hook: False launches sg_sparse_decode_attn fully ordered behind earlier work (no overlap of calls)."""
+    _lib.sg_testing_decode_overlap(1 if allowed else 0)
 
 
 def sg_testing_score_grid(shape: "Shape") -> int:

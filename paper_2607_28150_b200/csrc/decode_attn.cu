@@ -262,13 +262,11 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
     }
   }
 
-  // Everything above reads only the KV sources, the index lists and the prefix arrays, which are stable
-  // inputs of a decode step; q (and the outputs) are ordered after all earlier work in the stream.
-  // Only an L2 prefetch of the query rows is issued early: L2 is where writes of earlier kernels land, so the
-  // loads behind the wait see current data, and find it on chip when nobody rewrote it in between.
-  if (warp == 0 && lane * 64 < p.G * D)
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p.q + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D + lane * 64));
-  pdl_wait();
+  // Everything in this kernel up to its output stores reads only inputs of the decode step -- the KV sources, the
+  // index lists, the prefix arrays and the query rows -- which the contract treats as stable: they must not be
+  // written by a kernel that itself lets its dependents start early (such as the previous layer's call of this
+  // kernel).  So nothing waits here: the dependency wait sits in front of the stores of out / lse, and consecutive
+  // calls overlap everything but those stores.
   // Q fragments (A operand, 16 x D, rows >= G are zero).
   const int r_lo = lane >> 2, r_hi = r_lo + 8;
   uint32_t qa[D / 16][4];
@@ -437,6 +435,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
   __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(p.out) + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
   float* lsep = p.lse ? p.lse + (int64_t)b * p.Hq + (int64_t)g * p.G : nullptr;
   if (cs > 1) cluster_wait();                                  // every CTA of the cluster has started
+  if (cs == 1) pdl_wait();                                     // out / lse are written below: all earlier work in the stream first
   // two neighbouring outputs per thread (same row, same owner: D and the owners' slices are even)
   for (int e = 2 * tid; e < p.G * D; e += 2 * kDecThreads) {
     const int r = e / D, col = e - r * D;
@@ -473,6 +472,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, kDecWarps == 4 ? 2 : 1) decode
       raise(p.dev_status, SG_ERR_TIMEOUT);
       return;
     }
+    pdl_wait();                                                // out / lse are written below: all earlier work in the stream first
     for (int e = e_beg + tid; e < e_end; e += kDecThreads) {
       const int r = e / D, col = e - r * D;
       float mj[8], lj[8], oj[8];
@@ -547,6 +547,8 @@ size_t decode_workspace_bytes(const sg_shape*, int32_t, int32_t) { return 0; }  
 
 namespace sg {
 namespace {
+// Testing hook (sg_testing_decode_overlap): 0 launches the decode kernel fully ordered behind earlier work.
+std::atomic<int> g_test_decode_overlap{1};
 sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed_k, const void* packed_v, const int32_t* cu_k,
                         int32_t total_sel, const int32_t* packed_count, const int32_t* local_skip, const void* local_k,
                         const void* local_v, const int32_t* local_idx, const int32_t* cu_nloc, int32_t total_loc,
@@ -554,6 +556,10 @@ sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed
                         int32_t* dev_status, void* stream);
 }
 }  // namespace sg
+
+extern "C" void sg_testing_decode_overlap(int32_t allowed) {
+  sg::g_test_decode_overlap.store(allowed, std::memory_order_relaxed);
+}
 
 extern "C" sg_status sg_sparse_decode_attn(const sg_shape* shape, const void* q, const void* packed_k,
                                            const void* packed_v, const int32_t* cu_k, int32_t total_sel,
@@ -630,7 +636,7 @@ sg_status decode_launch(const sg_shape* shape, const void* q, const void* packed
 
   cudaLaunchAttribute attrs[2];
   attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attrs[0].val.programmaticStreamSerializationAllowed = 1;
+  attrs[0].val.programmaticStreamSerializationAllowed = g_test_decode_overlap.load(std::memory_order_relaxed) ? 1 : 0;
   attrs[1].id = cudaLaunchAttributeClusterDimension;
   attrs[1].val.clusterDim.x = (unsigned)p.csize;
   attrs[1].val.clusterDim.y = 1;
