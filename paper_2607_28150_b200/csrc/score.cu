@@ -46,7 +46,6 @@ constexpr int kMmaWarp = kTmaWarp + 1;
 constexpr int kHelperWarp = kTmaWarp + 2;
 constexpr int kScoreThreads = kEpiThreads + 128;
 constexpr int kTileKeys = 128;
-constexpr int kRing = 4 / kEpiGroups;        // accumulator stages per epilogue warpgroup
 constexpr int kAccStages = 4;             // 4 x 128 fp32 columns = the whole 512-column TMEM
 constexpr int kPartSlots = 8;             // pass 2, several row blocks per key tile: partial column sums of up to 8 tiles in flight
 constexpr uint32_t kTmemCols = 512;
@@ -72,6 +71,17 @@ constexpr int kClockWords = 32;
 constexpr int kClockWords = 4;
 #endif
 
+// Debug build (-DSG_CHECKS): device-side checks of the shared-memory carve-up, of every TMA coordinate (16-byte
+// aligned innermost coordinate, tile inside the tensor or hanging over its end only where the fill value is
+// wanted) and of every TMEM address against the allocation.  A failed check never traps: it sets the
+// SG_ERR_INVALID bit of the status word and the access is still made only if it is known to be harmless (TMA
+// loads past the end are zero-filled by the hardware), so a debug run ends like any other and reports the bit.
+#ifdef SG_CHECKS
+#define SG_CHECK(cond) do { if (!(cond)) raise(p.dev_status, SG_ERR_INVALID); } while (0)
+#else
+#define SG_CHECK(cond) do { } while (0)
+#endif
+
 struct ScoreParams {
   const int32_t* cu;
   float* importance;
@@ -84,6 +94,7 @@ struct ScoreParams {
   int32_t lag;             // pass 2 of unit u is scheduled `lag` units after its pass 1
   int32_t compact;         // schedule layout: 0 = every slot 2*C positions, 1 = positions without an item removed
   int32_t tiles_per_chunk, max_items, k_stages, q_bufs;
+  int32_t smem_bytes;      // dynamic shared memory of the launch (debug checks)
   int32_t wgslots;         // statistics slots per item: 4 (one per epilogue warpgroup) or 1 (every row block has one owner)
   int32_t withhold_unit;   // testing only: pass-1 items of this unit are never counted as done (-1 = none)
   uint32_t wait_ns;        // limit of every bounded wait, nanoseconds
@@ -157,26 +168,8 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem], bf16 x bf16 -> fp32, issued by one thread.  The operands are shared-memory
-// matrix descriptors given as their low words (address field); the high word is the same for every operand.
-template <bool kAccumulate>
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
-  if (kAccumulate) {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
-        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-        "setp.eq.u32 p, %1, %1;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
-        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-        "setp.ne.u32 p, %1, %1;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
-  }
-}
+// D[tmem] = A[smem] * B[smem], bf16 x bf16 -> fp32, issued by one thread; the operands are shared-memory matrix
+// descriptors given as their low words (address field), the high word is the same for every operand.
 // All MMAs of one accumulator block in a single statement: NK k-steps of 16 elements, four per 128-byte
 // sub-tile (descriptor low word += 2 per step inside a sub-tile, += a_sub / b_sub to the next sub-tile).  The first
 // MMA overwrites the accumulator, the others add to it.  One statement keeps the issuing thread's instruction
@@ -249,9 +242,6 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
     asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
                       "+r"(r[i + 6]), "+r"(r[i + 7]) :: "memory");
 }
-// Barrier among the 128 threads of one epilogue warpgroup (named barriers 2..5); no CTA-wide barrier is used
-// between the start and the end of the kernel.
-__device__ __forceinline__ void wg_bar_sync(int wg) { asm volatile("bar.sync %0, 128;" ::"r"(wg + 2) : "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
 // 128-byte swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B).  High word: 8-row groups are 1024
@@ -389,6 +379,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
   auto bar_stat_free = [&](int s) { return smem_u32(&bars[27 + s]); };   // helpers -> epilogue: the statistics buffer was published                        // MMA thread: every MMA it issued has completed
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    SG_CHECK(reinterpret_cast<uint8_t*>(s_prefix + p.B + 1) <= smem_dyn + p.smem_bytes);     // carve-up fits the launch's shared memory
+    SG_CHECK((smem_u32(q_smem) & 1023u) == 0 && (smem_u32(k_smem) & 1023u) == 0);            // swizzled operands on 1024-byte boundaries
+    SG_CHECK((smem_u32(bars) & 7u) == 0 && (smem_u32(lse_buf) & 15u) == 0);
+  }
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -470,6 +465,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         SG_PROF_ADD(w_qempty, tq);
         if (!ok) break;
         ++n_item;
+        SG_CHECK(qb >= 0 && qb < p.q_bufs && (it.g + 1) * p.G <= p.Hkv * p.G && it.b < p.B && p.G * p.W <= p.Ralloc);
         mbar_arrive_expect_tx(bar_qfull(qb), (uint32_t)(kSub * p.G * p.W * 128));
 #pragma unroll
         for (int dc = 0; dc < kSub; ++dc)
@@ -480,6 +476,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
           ok = mbar_wait(bar_kempty(stage), phase ^ 1u, abort_flag, p.wait_ns, 200u);
           SG_PROF_ADD(w_kempty, tk);
           if (!ok) break;
+          SG_CHECK(stage >= 0 && stage < p.k_stages && it.c0 + tile * kTileKeys < p.T && it.g < p.Hkv && it.l * p.Hkv < p.U);
           mbar_arrive_expect_tx(bar_kfull(stage), (uint32_t)kKStageBytes);
 #pragma unroll
           for (int dc = 0; dc < kSub; ++dc)
@@ -590,6 +587,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     // log-sum-exps, so the others keep the SFU busy while one of them is between items.
     const int wg = warp >> 2;
     const int wg_tid = tid & 127;
+    (void)wg_tid;                                      // only the profiling build reads it
     const int lane_grp = warp & 3;                     // TMEM lane quarter this warp may access
     const int row_in_tile = lane_grp * 32 + lane;
     const uint32_t t_lane = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
@@ -708,6 +706,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             uint32_t cur[32];
 #pragma unroll 1
             for (int j = 0; j < 4; ++j) {
+              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
               tmem_ld_wait(cur);
               if (j == 3) release_acc();
@@ -779,6 +778,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             uint32_t cur[32];
 #pragma unroll 1
             for (int j = 0; j < nchk; ++j) {
+              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
               tmem_ld_wait(cur);
               if (j == nchk - 1) release_acc();
@@ -810,6 +810,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             __syncwarp();
             if (lane == 0) sm_cnt[slot * 4 + lane_grp] = 0;
           }
+          SG_CHECK(!(ok && t < N) || (it.c0 + t < p.T && it.l * p.Hkv + it.g < p.U));
           if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
         }
         __syncwarp();
@@ -1167,6 +1168,7 @@ extern "C" sg_status sg_score(const sg_shape* shape, const void* q_win, const vo
   p.max_items = pl.max_items;
   p.k_stages = pl.k_stages;
   p.q_bufs = pl.q_bufs;
+  p.smem_bytes = pl.smem_bytes;
   p.wgslots = pl.wgslots;
   p.withhold_unit = g_test_withhold_unit.load(std::memory_order_relaxed);
   const int limit_ms = g_test_wait_limit_ms.load(std::memory_order_relaxed);

@@ -103,3 +103,19 @@ int main(void) {
                     "-L", libdir, "-lsmartgen", "-Wl,-rpath," + libdir], check=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout
     assert "c caller ok" in out
+
+
+def test_debug_and_profiling_builds_of_the_scoring_kernel_compile(tmp_path):
+    """The library has two optional builds of csrc/score.cu (SG_NVCC_FLAGS of the build script): -DSG_CHECKS adds
+    device-side checks of shared-memory carve-up, TMA coordinates and TMEM addresses that report through the status
+    word and never trap; -DSG_SCORE_PROFILE adds per-role wait counters.  Both must keep compiling for sm_100a."""
+    import shutil
+    import subprocess
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        return
+    src = os.path.join(ROOT, "paper_2607_28150_b200", "csrc", "score.cu")
+    for flag in ("-DSG_CHECKS", "-DSG_SCORE_PROFILE"):
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O1", "-std=c++17", "--use_fast_math", flag,
+                        "-I", os.path.join(ROOT, "include"), "-I", os.path.dirname(src), "-c", src,
+                        "-o", str(tmp_path / "score_dbg.o")], check=True, capture_output=True)
