@@ -342,6 +342,26 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* ptr) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
   return v;
 }
+// Rare path of pass 1: the sum of a 32-column chunk against the running reference m left the safe range (a value far
+// above m, or m still -inf at the start of a work item).  Takes the chunk's maximum, rescales the running sum and adds
+// the chunk against the new reference.  Kept out of line so that the hot loop holds nothing but its 32 x (fma, ex2, add).
+// (Everything is passed and returned by value: taking the address of the chunk's registers or of the running statistics
+// would move them to local memory in the hot loop as well.)
+__device__ __noinline__ float2 refresh_reference(float scale_log2, float m, float lsum, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t c4, uint32_t c5, uint32_t c6, uint32_t c7, uint32_t c8, uint32_t c9, uint32_t c10, uint32_t c11, uint32_t c12, uint32_t c13, uint32_t c14, uint32_t c15, uint32_t c16, uint32_t c17, uint32_t c18, uint32_t c19, uint32_t c20, uint32_t c21, uint32_t c22, uint32_t c23, uint32_t c24, uint32_t c25, uint32_t c26, uint32_t c27, uint32_t c28, uint32_t c29, uint32_t c30, uint32_t c31) {
+  const uint32_t cur[32] = {c0, c1, c2, c3, c4, c5, c6, c7, c8, c9, c10, c11, c12, c13, c14, c15, c16, c17, c18, c19, c20, c21, c22, c23, c24, c25, c26, c27, c28, c29, c30, c31};
+  float mx = __uint_as_float(cur[0]);
+#pragma unroll
+  for (int c = 1; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(cur[c]));
+  const float mn = fmaxf(m, mx * scale_log2);
+  float r0 = 0.f, r1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 32; c += 2) {
+    r0 += exp2f(fmaf(__uint_as_float(cur[c]), scale_log2, -mn));
+    r1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), scale_log2, -mn));
+  }
+  return make_float2(mn, lsum * exp2f(m - mn) + (r0 + r1));
+}
+
 template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, const ScoreParams p) {
@@ -653,14 +673,21 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const bool row_ok = r < p.R && (r / p.G) < Weff;
             const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
             float m = sm_m[r], lsum = sm_l[r];
-            // one 32-column chunk of this thread's row: online (max, sum of exp2) in the log2 domain
-            auto chunk = [&](const uint32_t (&cur)[32], const int col0) {
-              if (all_visible && row_ok) {
-                // The running reference m need not be the row maximum: fp32 keeps its relative precision for any
-                // exponent, so the sum of exp2(x - m) is as accurate with a stale (lower) m as with the true maximum,
-                // as long as nothing overflows.  The chunk is therefore summed against the current m first (no
-                // maximum over its 32 values); only if the sum leaves the safe range -- a value more than ~60 binary
-                // orders above m, or m still -inf at the start of an item -- is the maximum taken and the chunk redone.
+            uint32_t cur[32];
+            if (all_visible && __all_sync(0xffffffffu, row_ok)) {
+              // Hot loop: every key of the tile is visible to every row of the warp.  The running reference m need not
+              // be the row maximum: fp32 keeps its relative precision for any exponent, so the sum of exp2(x - m) is as
+              // accurate with a stale (lower) m as with the true maximum, as long as nothing overflows.  A chunk is
+              // summed against the current m (no maximum over its 32 values); only if the sum leaves the safe range -- a
+              // value more than ~60 binary orders above m, or m still -inf at the start of an item -- is the reference
+              // refreshed, out of line.  The loop body is 32 x (fma, ex2, add) and nothing else: with the masked
+              // variants compiled into the same body it ran 11-15 % slower.
+#pragma unroll 1
+              for (int j = 0; j < 4; ++j) {
+                SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
+                tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+                tmem_ld_wait(cur);
+                if (j == 3) release_acc();
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 32; c += 4) {
@@ -670,47 +697,30 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                   s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -m));
                 }
                 const float s = (s0 + s1) + (s2 + s3);
-                if (s < 0x1p60f) {
-                  lsum += s;
-                } else {
-                  float mx0 = __uint_as_float(cur[0]), mx1 = __uint_as_float(cur[1]);
-                  float mx2 = __uint_as_float(cur[2]), mx3 = __uint_as_float(cur[3]);
+                if (s < 0x1p60f) lsum += s;
+                else { const float2 ml = refresh_reference(p.scale_log2, m, lsum, cur[0], cur[1], cur[2], cur[3], cur[4], cur[5], cur[6], cur[7], cur[8], cur[9], cur[10], cur[11], cur[12], cur[13], cur[14], cur[15], cur[16], cur[17], cur[18], cur[19], cur[20], cur[21], cur[22], cur[23], cur[24], cur[25], cur[26], cur[27], cur[28], cur[29], cur[30], cur[31]); m = ml.x; lsum = ml.y; }
+              }
+            } else {
+              // Tile on the causal diagonal, or rows outside the window in this warp: per-column masks, true maximum.
+#pragma unroll 1
+              for (int j = 0; j < 4; ++j) {
+                const int col0 = j * 32;
+                tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
+                tmem_ld_wait(cur);
+                if (j == 3) release_acc();
+                if (col0 <= cmax) {
+                  float mx = -INFINITY;
 #pragma unroll
-                  for (int c = 4; c < 32; c += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(cur[c]));     mx1 = fmaxf(mx1, __uint_as_float(cur[c + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(cur[c + 2])); mx3 = fmaxf(mx3, __uint_as_float(cur[c + 3]));
-                  }
-                  const float mn = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
-                  float r0 = 0.f, r1 = 0.f;
+                  for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, __uint_as_float(cur[c])) : mx;
+                  const float mn = fmaxf(m, mx * p.scale_log2);
+                  float s = 0.f;
 #pragma unroll
-                  for (int c = 0; c < 32; c += 2) {
-                    r0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn));
-                    r1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -mn));
-                  }
-                  lsum = lsum * exp2f(m - mn) + (r0 + r1);
+                  for (int c = 0; c < 32; ++c)
+                    s += (col0 + c <= cmax) ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn)) : 0.f;
+                  lsum = lsum * exp2f(m - mn) + s;
                   m = mn;
                 }
-              } else if (col0 <= cmax) {
-                float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, __uint_as_float(cur[c])) : mx;
-                const float mn = fmaxf(m, mx * p.scale_log2);
-                float s = 0.f;
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                  s += (col0 + c <= cmax) ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn)) : 0.f;
-                lsum = lsum * exp2f(m - mn) + s;
-                m = mn;
               }
-            };
-            uint32_t cur[32];
-#pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
-              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
-              tmem_ld_wait(cur);
-              if (j == 3) release_acc();
-              chunk(cur, j * 32);
             }
             sm_m[r] = m;
             sm_l[r] = lsum;
@@ -755,10 +765,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             tc_fence_after();
             const int ncols = min(128, p.Rpad - blk * 128);
             const int nchk = (ncols + 31) >> 5;          // 32-column chunks of this block (warp-uniform)
-            // one 32-column chunk of this thread's key: add exp2(s*c - lse_r) over the visible query rows
-            auto chunk = [&](const uint32_t (&cur)[32], const int col0) {
-              const float* ls = lse2 + blk * 128 + col0;
-              if (all_visible && col0 + 32 <= ncols) {
+            uint32_t cur[32];
+            if (all_visible && ncols == 128) {
+              // Hot loop: every row of the block sees every key of the tile; nothing but 32 x (fma, ex2, add) and the
+              // rows' log-sum-exps from shared memory.
+#pragma unroll 1
+              for (int j = 0; j < 4; ++j) {
+                SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
+                tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+                tmem_ld_wait(cur);
+                if (j == 3) release_acc();
+                const float* ls = lse2 + blk * 128 + j * 32;
 #pragma unroll
                 for (int c = 0; c < 32; c += 4) {
                   const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
@@ -767,22 +784,22 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                   a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
                   a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
                 }
-              } else {
+              }
+            } else {
+              // Tile on the causal diagonal, or a partial last row block: per-column masks.
+#pragma unroll 1
+              for (int j = 0; j < nchk; ++j) {
+                const int col0 = j * 32;
+                tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
+                tmem_ld_wait(cur);
+                if (j == nchk - 1) release_acc();
+                const float* ls = lse2 + blk * 128 + col0;
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                   const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
                   a0 += vis ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -ls[c])) : 0.f;
                 }
               }
-            };
-            uint32_t cur[32];
-#pragma unroll 1
-            for (int j = 0; j < nchk; ++j) {
-              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
-              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
-              tmem_ld_wait(cur);
-              if (j == nchk - 1) release_acc();
-              chunk(cur, j * 32);
             }
           }
           float total = (a0 + a1) + (a2 + a3);
