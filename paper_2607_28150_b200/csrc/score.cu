@@ -657,7 +657,59 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             sm_m[blk * 128 + row_in_tile] = -INFINITY;
             sm_l[blk * 128 + row_in_tile] = 0.f;
           }
-        for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
+        // The item's tiles in two loops.  First the tiles that every window row sees completely, when all rows of this
+        // warp lie inside the window: the loop holds the hot body and nothing else -- with the masked variant compiled
+        // into the same loop the kernel, which runs at its 96-register limit, was 7-10 % slower as a whole.  Then the
+        // rest (the causal diagonal, or everything when some row of the warp is outside the window) in the general loop.
+        bool rows_ok = true;
+        for (int blk = 0; blk < nblk; ++blk) {
+          const int r = blk * 128 + row_in_tile;
+          rows_ok = rows_ok && r < p.R && (r / p.G) < Weff;
+        }
+        rows_ok = __all_sync(0xffffffffu, rows_ok);
+        const int vis_end = (first_win + 1) / kTileKeys;                    // tiles [0, vis_end) are visible to every window row
+        const int hot_end = rows_ok ? min(it.tile_end, max(it.tile_beg, vis_end)) : it.tile_beg;
+        for (int tile = it.tile_beg; tile < hot_end; ++tile) {
+          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+          for (int blk = 0; blk < nblk; ++blk) {
+            if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+            SG_PROF_BEGIN(ta);
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
+            SG_PROF_ADD(w_afull, ta);
+            SG_PROF_INC(n_blocks);
+            if (!ok) continue;
+            tc_fence_after();
+            const int r = blk * 128 + row_in_tile;
+            float m = sm_m[r], lsum = sm_l[r];
+            uint32_t cur[32];
+            // The running reference m need not be the row maximum: fp32 keeps its relative precision for any exponent, so
+            // the sum of exp2(x - m) is as accurate with a stale (lower) m as with the true maximum, as long as nothing
+            // overflows.  A chunk is summed against the current m (no maximum over its 32 values); only if the sum leaves
+            // the safe range -- a value more than ~60 binary orders above m, or m still -inf at the start of an item --
+            // is the reference refreshed, out of line.  The loop body is 32 x (fma, ex2, add) and nothing else.
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
+              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+              tmem_ld_wait(cur);
+              if (j == 3) release_acc();
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; c += 4) {
+                s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -m));
+                s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -m));
+                s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -m));
+                s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -m));
+              }
+              const float s = (s0 + s1) + (s2 + s3);
+              if (s < 0x1p60f) lsum += s;
+              else { const float2 ml = refresh_reference(p.scale_log2, m, lsum, cur[0], cur[1], cur[2], cur[3], cur[4], cur[5], cur[6], cur[7], cur[8], cur[9], cur[10], cur[11], cur[12], cur[13], cur[14], cur[15], cur[16], cur[17], cur[18], cur[19], cur[20], cur[21], cur[22], cur[23], cur[24], cur[25], cur[26], cur[27], cur[28], cur[29], cur[30], cur[31]); m = ml.x; lsum = ml.y; }
+            }
+            sm_m[r] = m;
+            sm_l[r] = lsum;
+          }
+        }
+        for (int tile = hot_end; tile < it.tile_end; ++tile) {
           if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t0 = tile * kTileKeys;
           const bool all_visible = t0 + kTileKeys - 1 <= first_win;
@@ -746,7 +798,78 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         if (ok) ok = mbar_wait(bar_lse_ready(lbuf), lph, abort_flag, p.wait_ns, 32u);
         SG_PROF_ADD(w_lse, tl);
         const float* lse2 = lse_buf + lbuf * p.Ralloc;   // [Ralloc] row log-sum-exps (log2 domain) of (unit, b)
-        for (int tile = it.tile_beg; tile < it.tile_end; ++tile) {
+        // End of a tile for this warp: its partial (or whole) column sum goes out.
+        auto finish_tile = [&](const int tile, const int t, const float a0, const float a1, const float a2, const float a3, const uint32_t n0,
+                               const bool mine) {
+          float total = (a0 + a1) + (a2 + a3);
+          if (blockwise) {
+            // The tile's row blocks were dealt to different warpgroups.  Each warpgroup that had one leaves its partial
+            // column sums in shared memory; per lane quarter, the warp that writes the last partial adds them up in a
+            // fixed order (bitwise reproducible) and stores the importance -- no block-wide barrier per tile.  A slot
+            // is reused S tiles later: block m is issued only after blocks m-4 .. m-7 were released, and the
+            // warpgroups that released them had finished everything up to block m-8; with (S-1)*nblk >= 7 all
+            // partials of the slot's previous tile are summed before the slot is written again.
+            if (!mine) return;
+            const int nwg = nblk < kEpiGroups ? nblk : kEpiGroups;      // warpgroups that drain blocks of this tile
+            const int slot = tile & (nblk >= 4 ? 3 : 7);
+            float* part = sm_part + slot * (kEpiGroups * 128);
+            part[wg * 128 + row_in_tile] = total;
+            __threadfence_block();
+            __syncwarp();
+            int old = 0;
+            if (lane == 0) old = atomicAdd(&sm_cnt[slot * 4 + lane_grp], 1);
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if (old != nwg - 1) return;
+            __threadfence_block();
+            total = 0.f;
+            for (int i = 0; i < nwg; ++i) total += part[((n0 + i) % kEpiGroups) * 128 + row_in_tile];
+            __syncwarp();
+            if (lane == 0) sm_cnt[slot * 4 + lane_grp] = 0;
+          }
+          SG_CHECK(!(ok && t < N) || (it.c0 + t < p.T && it.l * p.Hkv + it.g < p.U));
+          if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
+        };
+        // Two loops, as in pass 1: the tiles every window row sees completely, when every row block is full (hot body
+        // only), then the rest in the general loop.
+        const int vis_end = (first_win + 1) / kTileKeys;
+        const int hot_end = (p.Rpad & 127) == 0 ? min(it.tile_end, max(it.tile_beg, vis_end)) : it.tile_beg;
+        for (int tile = it.tile_beg; tile < hot_end; ++tile) {
+          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+          const int t = tile * kTileKeys + row_in_tile;  // this thread's key
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          const uint32_t n0 = tile_count;                // running block count at the start of this tile
+          bool mine = false;                             // this warpgroup drains at least one block of the tile
+          for (int blk = 0; blk < nblk; ++blk) {
+            if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+            mine = true;
+            SG_PROF_BEGIN(ta);
+            if (ok) ok = mbar_wait(bar_afull(as), aph, abort_flag, p.wait_ns, 0u);
+            SG_PROF_ADD(w_afull, ta);
+            SG_PROF_INC(n_blocks);
+            if (!ok) continue;
+            tc_fence_after();
+            uint32_t cur[32];
+            // nothing but 32 x (fma, ex2, add) and the rows' log-sum-exps from shared memory
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+              SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
+              tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
+              tmem_ld_wait(cur);
+              if (j == 3) release_acc();
+              const float* ls = lse2 + blk * 128 + j * 32;
+#pragma unroll
+              for (int c = 0; c < 32; c += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
+                a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
+                a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
+                a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
+              }
+            }
+          }
+          finish_tile(tile, t, a0, a1, a2, a3, n0, mine);
+        }
+        for (int tile = hot_end; tile < it.tile_end; ++tile) {
           if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
           const int t = tile * kTileKeys + row_in_tile;  // this thread's key
           const bool all_visible = tile * kTileKeys + kTileKeys - 1 <= first_win;
@@ -802,33 +925,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
               }
             }
           }
-          float total = (a0 + a1) + (a2 + a3);
-          if (blockwise) {
-            // The tile's row blocks were dealt to different warpgroups.  Each warpgroup that had one leaves its partial
-            // column sums in shared memory; per lane quarter, the warp that writes the last partial adds them up in a
-            // fixed order (bitwise reproducible) and stores the importance -- no block-wide barrier per tile.  A slot
-            // is reused S tiles later: block m is issued only after blocks m-4 .. m-7 were released, and the
-            // warpgroups that released them had finished everything up to block m-8; with (S-1)*nblk >= 7 all
-            // partials of the slot's previous tile are summed before the slot is written again.
-            if (!mine) continue;
-            const int nwg = nblk < kEpiGroups ? nblk : kEpiGroups;      // warpgroups that drain blocks of this tile
-            const int slot = tile & (nblk >= 4 ? 3 : 7);
-            float* part = sm_part + slot * (kEpiGroups * 128);
-            part[wg * 128 + row_in_tile] = total;
-            __threadfence_block();
-            __syncwarp();
-            int old = 0;
-            if (lane == 0) old = atomicAdd(&sm_cnt[slot * 4 + lane_grp], 1);
-            old = __shfl_sync(0xffffffffu, old, 0);
-            if (old != nwg - 1) continue;
-            __threadfence_block();
-            total = 0.f;
-            for (int i = 0; i < nwg; ++i) total += part[((n0 + i) % kEpiGroups) * 128 + row_in_tile];
-            __syncwarp();
-            if (lane == 0) sm_cnt[slot * 4 + lane_grp] = 0;
-          }
-          SG_CHECK(!(ok && t < N) || (it.c0 + t < p.T && it.l * p.Hkv + it.g < p.U));
-          if (ok && t < N) p.importance[((size_t)it.l * p.Hkv + it.g) * p.T + it.c0 + t] = total;
+          finish_tile(tile, t, a0, a1, a2, a3, n0, mine);
         }
         __syncwarp();
         if (lane == 0 && ok) mbar_arrive(bar_lse_free(lbuf));        // this warp no longer reads lse_buf[lbuf]
