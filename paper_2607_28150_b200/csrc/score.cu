@@ -726,53 +726,34 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const int cmax = row_ok ? (first_win + r / p.G - t0) : -1;    // last visible column of this tile
             float m = sm_m[r], lsum = sm_l[r];
             uint32_t cur[32];
-            if (all_visible && __all_sync(0xffffffffu, row_ok)) {
-              // Hot loop: every key of the tile is visible to every row of the warp.  The running reference m need not
-              // be the row maximum: fp32 keeps its relative precision for any exponent, so the sum of exp2(x - m) is as
-              // accurate with a stale (lower) m as with the true maximum, as long as nothing overflows.  A chunk is
-              // summed against the current m (no maximum over its 32 values); only if the sum leaves the safe range -- a
-              // value more than ~60 binary orders above m, or m still -inf at the start of an item -- is the reference
-              // refreshed, out of line.  The loop body is 32 x (fma, ex2, add) and nothing else: with the masked
-              // variants compiled into the same body it ran 11-15 % slower.
+            // Chunk by chunk: where every row of the warp sees all 32 keys of the chunk (all but the last chunk or two
+            // of a tile on the causal diagonal, and every chunk of a fully visible tile) the hot body, else per-column
+            // masks with the true maximum.  (all_visible enters only to spare the vote on fully visible tiles.)
 #pragma unroll 1
-              for (int j = 0; j < 4; ++j) {
-                SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
-                tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
-                tmem_ld_wait(cur);
-                if (j == 3) release_acc();
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            for (int j = 0; j < 4; ++j) {
+              const int col0 = j * 32;
+              SG_CHECK(as * 128 + col0 + 32 <= (int)kTmemCols);
+              tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
+              tmem_ld_wait(cur);
+              if (j == 3) release_acc();
+              if (!__all_sync(0xffffffffu, row_ok && (all_visible || col0 + 31 <= cmax))) {
+                // Some (row, key) pairs of the chunk are hidden: a thread that sees nothing of it is done; the others
+                // replace their hidden scores by -inf, which the body below ignores (exp2 of it is 0, no maximum takes it).
+                if (col0 > cmax) continue;
 #pragma unroll
-                for (int c = 0; c < 32; c += 4) {
-                  s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -m));
-                  s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -m));
-                  s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -m));
-                  s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -m));
-                }
-                const float s = (s0 + s1) + (s2 + s3);
-                if (s < 0x1p60f) lsum += s;
-                else { const float2 ml = refresh_reference(p.scale_log2, m, lsum, cur[0], cur[1], cur[2], cur[3], cur[4], cur[5], cur[6], cur[7], cur[8], cur[9], cur[10], cur[11], cur[12], cur[13], cur[14], cur[15], cur[16], cur[17], cur[18], cur[19], cur[20], cur[21], cur[22], cur[23], cur[24], cur[25], cur[26], cur[27], cur[28], cur[29], cur[30], cur[31]); m = ml.x; lsum = ml.y; }
+                for (int c = 0; c < 32; ++c) cur[c] = (col0 + c <= cmax) ? cur[c] : 0xff800000u;
               }
-            } else {
-              // Tile on the causal diagonal, or rows outside the window in this warp: per-column masks, true maximum.
-#pragma unroll 1
-              for (int j = 0; j < 4; ++j) {
-                const int col0 = j * 32;
-                tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
-                tmem_ld_wait(cur);
-                if (j == 3) release_acc();
-                if (col0 <= cmax) {
-                  float mx = -INFINITY;
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                  for (int c = 0; c < 32; ++c) mx = (col0 + c <= cmax) ? fmaxf(mx, __uint_as_float(cur[c])) : mx;
-                  const float mn = fmaxf(m, mx * p.scale_log2);
-                  float s = 0.f;
-#pragma unroll
-                  for (int c = 0; c < 32; ++c)
-                    s += (col0 + c <= cmax) ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -mn)) : 0.f;
-                  lsum = lsum * exp2f(m - mn) + s;
-                  m = mn;
-                }
+              for (int c = 0; c < 32; c += 4) {
+                s0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -m));
+                s1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -m));
+                s2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -m));
+                s3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -m));
               }
+              const float s = (s0 + s1) + (s2 + s3);
+              if (s < 0x1p60f) lsum += s;      // false also for the NaN that a hidden score gives while m is still -inf
+              else { const float2 ml = refresh_reference(p.scale_log2, m, lsum, cur[0], cur[1], cur[2], cur[3], cur[4], cur[5], cur[6], cur[7], cur[8], cur[9], cur[10], cur[11], cur[12], cur[13], cur[14], cur[15], cur[16], cur[17], cur[18], cur[19], cur[20], cur[21], cur[22], cur[23], cur[24], cur[25], cur[26], cur[27], cur[28], cur[29], cur[30], cur[31]); m = ml.x; lsum = ml.y; }
             }
             sm_m[r] = m;
             sm_l[r] = lsum;
@@ -889,39 +870,35 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const int ncols = min(128, p.Rpad - blk * 128);
             const int nchk = (ncols + 31) >> 5;          // 32-column chunks of this block (warp-uniform)
             uint32_t cur[32];
-            if (all_visible && ncols == 128) {
-              // Hot loop: every row of the block sees every key of the tile; nothing but 32 x (fma, ex2, add) and the
-              // rows' log-sum-exps from shared memory.
+            // Chunk by chunk: where all 32 rows of the chunk exist and see every key of the warp (on the causal diagonal:
+            // all warps but the one that holds the window's own keys) the hot body, else per-column masks.
 #pragma unroll 1
-              for (int j = 0; j < 4; ++j) {
-                SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
-                tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
-                tmem_ld_wait(cur);
-                if (j == 3) release_acc();
-                const float* ls = lse2 + blk * 128 + j * 32;
+            for (int j = 0; j < nchk; ++j) {
+              const int col0 = j * 32;
+              SG_CHECK(as * 128 + col0 + 32 <= (int)kTmemCols && blk * 128 + col0 + 32 <= p.Ralloc);
+              tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
+              tmem_ld_wait(cur);
+              if (j == nchk - 1) release_acc();
+              const float* ls = lse2 + blk * 128 + col0;
+              if (!(col0 + 32 <= ncols && (all_visible || __all_sync(0xffffffffu, blk * 128 + col0 >= rmin)))) {
+                // rows that do not see this thread's key (those below c_lo of this chunk), or that do not exist (from c_hi
+                // on, in a partial last chunk): score -inf, probability 0
+                const int c_lo = rmin - blk * 128 - col0, c_hi = ncols - col0;
+                if (c_hi >= 32) {
 #pragma unroll
-                for (int c = 0; c < 32; c += 4) {
-                  const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
-                  a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
-                  a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
-                  a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
-                  a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
+                  for (int c = 0; c < 32; ++c) cur[c] = c >= c_lo ? cur[c] : 0xff800000u;
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 32; ++c) cur[c] = (c >= c_lo && c < c_hi) ? cur[c] : 0xff800000u;
                 }
               }
-            } else {
-              // Tile on the causal diagonal, or a partial last row block: per-column masks.
-#pragma unroll 1
-              for (int j = 0; j < nchk; ++j) {
-                const int col0 = j * 32;
-                tmem_ld32_issue(cur, t_acc + (uint32_t)col0);
-                tmem_ld_wait(cur);
-                if (j == nchk - 1) release_acc();
-                const float* ls = lse2 + blk * 128 + col0;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                  const bool vis = (col0 + c < ncols) && (blk * 128 + col0 + c >= rmin);
-                  a0 += vis ? exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -ls[c])) : 0.f;
-                }
+              for (int c = 0; c < 32; c += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(ls + c);
+                a0 += exp2f(fmaf(__uint_as_float(cur[c]), p.scale_log2, -l4.x));
+                a1 += exp2f(fmaf(__uint_as_float(cur[c + 1]), p.scale_log2, -l4.y));
+                a2 += exp2f(fmaf(__uint_as_float(cur[c + 2]), p.scale_log2, -l4.z));
+                a3 += exp2f(fmaf(__uint_as_float(cur[c + 3]), p.scale_log2, -l4.w));
               }
             }
           }
