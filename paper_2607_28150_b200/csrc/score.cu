@@ -670,7 +670,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int vis_end = (first_win + 1) / kTileKeys;                    // tiles [0, vis_end) are visible to every window row
         const int hot_end = rows_ok ? min(it.tile_end, max(it.tile_beg, vis_end)) : it.tile_beg;
         for (int tile = it.tile_beg; tile < hot_end; ++tile) {
-          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+          if (!blockwise && ((tile_count++) % kEpiGroups) != (uint32_t)wg) continue;   // (the wait below looks at `ok`)
           for (int blk = 0; blk < nblk; ++blk) {
             if (blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
             SG_PROF_BEGIN(ta);
@@ -687,7 +687,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             // overflows.  A chunk is summed against the current m (no maximum over its 32 values); only if the sum leaves
             // the safe range -- a value more than ~60 binary orders above m, or m still -inf at the start of an item --
             // is the reference refreshed, out of line.  The loop body is 32 x (fma, ex2, add) and nothing else.
-#pragma unroll 1
+#pragma unroll 2   // measured: 1, 2 and 4 give 685 / 667 / 680 us on the long-context shape
             for (int j = 0; j < 4; ++j) {
               SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols);
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
@@ -815,7 +815,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int vis_end = (first_win + 1) / kTileKeys;
         const int hot_end = (p.Rpad & 127) == 0 ? min(it.tile_end, max(it.tile_beg, vis_end)) : it.tile_beg;
         for (int tile = it.tile_beg; tile < hot_end; ++tile) {
-          if (!blockwise && (((tile_count++) % kEpiGroups) != (uint32_t)wg || !ok)) continue;
+          if (!blockwise && ((tile_count++) % kEpiGroups) != (uint32_t)wg) continue;   // (the wait below looks at `ok`)
           const int t = tile * kTileKeys + row_in_tile;  // this thread's key
           float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
           const uint32_t n0 = tile_count;                // running block count at the start of this tile
@@ -831,7 +831,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             tc_fence_after();
             uint32_t cur[32];
             // nothing but 32 x (fma, ex2, add) and the rows' log-sum-exps from shared memory
-#pragma unroll 1
+#pragma unroll 2
             for (int j = 0; j < 4; ++j) {
               SG_CHECK(as * 128 + j * 32 + 32 <= (int)kTmemCols && blk * 128 + j * 32 + 32 <= p.Ralloc);
               tmem_ld32_issue(cur, t_acc + (uint32_t)(j * 32));
