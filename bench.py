@@ -43,7 +43,7 @@ UNIT = "GB/s"
 NCU_TRAFFIC = {
     # captured on 8 of the 32 layers: per-launch bytes scaled x4 where a launch
     # covers all layers; the decode call is per layer.  (pack: its stores were still in L2 when the capture ended.)
-    "c2": {"score": 4 * (140.738e6 + 6.275e6), "select": 4 * 2.125e6, "pack": 4 * (27.097e6 + 0.131e6),
+    "c2": {"score": 4 * (142.152e6 + 6.255e6), "select": 4 * 2.125e6, "pack": 4 * (27.097e6 + 0.131e6),
            "select_pack": (32 / 24) * (86.950e6 + 27.208e6), "decode": 5.146e6},
 }
 
